@@ -1,0 +1,165 @@
+/*
+ * mona.h — C ABI of the B200 (sm_100a) implementation of the MONA matrix-optimizer step.
+ *
+ * One call of mona_step() performs, for every 2-D weight of a parameter set, the loop body of
+ * Algorithm 1 ("MONA Optimizer"):
+ *
+ *     D_k  = G_k - G_{k-1}                         (Eq. alto_diff,   Algorithm 1 line 4)
+ *     A_k  = beta_a A_{k-1} + (1 - beta_a) D_k     (Eq. alto_accel,  line 5)
+ *     G~_k = G_k + alpha A_k                       (Eq. alto_grad,   line 6)
+ *     M_k  = mu M_{k-1} + G~_k                     (Eq. muon_momentum, line 7)
+ *     O_k  = Newton-Schulz(M_k, T)                 (Eq. newton_schulz, line 8)
+ *     W   <- W - eta (gamma O_k + lambda W)        (Eq. muon_update,   line 9)
+ *     G_{k-1} <- G_k                               (line 10)
+ *
+ * with X_0 = M_k / (||M_k||_F + eps), X_{t+1} = a X_t + b X_t X_t^T X_t + c X_t X_t^T X_t X_t^T X_t,
+ * and gamma = 0.2 sqrt(max(m, n)) unless overridden.
+ *
+ * Conventions
+ *   - All matrix pointers are DEVICE pointers unless a parameter says "host".  Arrays of pointers
+ *     (params, grads) and all structs are HOST memory.
+ *   - Matrices are row-major with leading dimension = cols.  Parameters are fp32 master weights;
+ *     gradients are fp32 or bf16 (per descriptor).
+ *   - The caller owns parameters, gradients, the state block and the workspace.  The handle owns only
+ *     small host/device tables, one internal stream and a few events.
+ *   - Every function returns a mona_status; nothing throws or aborts.  Problems detected on the device
+ *     (non-finite norm, a wait that ran out) are latched in a status word read by mona_poll_status().
+ *   - There is no CPU fallback: on a machine without an sm_100 device mona_create() fails with
+ *     MONA_ERR_ARCH / MONA_ERR_CUDA.
+ *   - One handle is used from one host thread and one stream at a time.
+ */
+#ifndef MONA_H_
+#define MONA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MONA_OK = 0,
+    MONA_ERR_INVALID_ARG = 1,        /* null pointer, non-positive size, bad enum                     */
+    MONA_ERR_UNSUPPORTED_SHAPE = 2,  /* a shape this build cannot process                             */
+    MONA_ERR_ALIGNMENT = 3,          /* a device pointer or stride is not 16-byte aligned             */
+    MONA_ERR_CUDA = 4,               /* a CUDA runtime/driver call failed (see mona_last_error)       */
+    MONA_ERR_TIMEOUT = 5,            /* a bounded device-side wait ran out                            */
+    MONA_ERR_NONFINITE = 6,          /* ||M_k||_F of some matrix was inf/nan                          */
+    MONA_ERR_ARCH = 7,               /* device is not compute capability 10.x                         */
+    MONA_ERR_BUFFER_TOO_SMALL = 8    /* state or workspace smaller than mona_query_sizes() reports    */
+} mona_status;
+
+typedef enum { MONA_F32 = 0, MONA_BF16 = 1 } mona_dtype;
+
+/* One descriptor = `batch` matrices of identical shape (the experts of one MoE layer, or batch = 1).
+ * Matrix b of the descriptor starts `b * batch_stride` ELEMENTS after the descriptor's base pointer,
+ * for the parameter and for the gradient alike.  The update scale gamma uses max(rows, cols) of one
+ * matrix, never the stacked shape. */
+typedef struct {
+    int64_t rows, cols;        /* m, n of one matrix                                                  */
+    int64_t batch;             /* >= 1                                                                */
+    int64_t batch_stride;      /* elements between consecutive matrices, >= rows*cols (0 = rows*cols) */
+    int32_t grad_dtype;        /* mona_dtype of the gradient                                          */
+    int32_t reserved;
+} mona_matrix_desc;
+
+/* REQUIRE line of Algorithm 1.  Doubles on purpose: (1 - beta_a), eta*gamma and eta*lambda are formed
+ * in double on the host and rounded to fp32 once. */
+typedef struct {
+    double lr;             /* eta                                                                     */
+    double momentum;       /* mu                                                                      */
+    double accel_beta;     /* beta_a                                                                  */
+    double accel_alpha;    /* alpha                                                                   */
+    double weight_decay;   /* lambda                                                                  */
+    double ns_a, ns_b, ns_c;  /* quintic coefficients (3.4445, -4.7750, 2.0315 in the paper)         */
+    double norm_eps;       /* X_0 = M / (||M||_F + eps); the paper has no eps, 1e-7 is a safe default */
+    double scale_value;    /* see scale_mode                                                          */
+    int32_t ns_steps;      /* T >= 0 (5 in the paper); 0 means O = X_0                                */
+    int32_t scale_mode;    /* 0: gamma = scale_value * sqrt(max(m,n)); 1: gamma = scale_value         */
+    int32_t ns_precision;  /* 0: bf16 operands on the tensor cores, fp32 accumulate;
+                              1: fp32 validation mode (plain FMA, no tensor cores)                    */
+    int32_t reserved;
+} mona_hparams;
+
+typedef struct mona_handle mona_handle;
+
+/* Fills *hp with the paper's defaults where it states them (T = 5, the quintic coefficients, the 0.2
+ * scale rule, beta_a = 0.99 with alpha = -1/(2(1-beta_a))) and eta = 1e-3, mu = 0.95, lambda = 0.1,
+ * eps = 1e-7 where it does not. */
+mona_status mona_default_hparams(mona_hparams* hp);
+
+/* Tuning knob, process-wide: bytes of bf16 Newton-Schulz iterates (X_t, X_{t+1}, A_t, B_t) one chunk of
+ * same-shape matrices may hold.  A chunk goes through all 3T GEMMs of the iteration before the next one
+ * starts, so it should fit the L2 cache.  Default 48 MiB; at least 1 MiB.  Affects later calls of
+ * mona_query_sizes() and mona_create() only. */
+mona_status mona_set_chunk_budget(size_t bytes);
+
+/* Bytes the caller must provide for the optimizer state (M, A, G_prev: 3 fp32 per parameter,
+ * Algorithm 1 line 1) and for the Newton-Schulz workspace.  Host only; no device is touched. */
+mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc,
+                             size_t* state_bytes, size_t* workspace_bytes);
+
+/* Builds the plan (shape buckets, chunking, tile schedules, TMA descriptors) for `n_desc` descriptors
+ * on CUDA device `device`, binds the caller's state and workspace blocks (both 256-byte aligned device
+ * memory of at least the queried sizes) and zero-fills the state (M_0 = A_0 = G_0 = 0).
+ * Synchronises the device once.  *out receives the handle; destroy it with mona_destroy(). */
+mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc,
+                        void* state, size_t state_bytes, void* workspace, size_t workspace_bytes,
+                        int device);
+
+/* One optimizer step for all descriptors, enqueued on `stream` (a cudaStream_t passed as void*;
+ * NULL = the legacy default stream).  params[i] / grads[i] are the device base pointers of
+ * descriptor i (16-byte aligned).  Reads grads, updates params and the state in place.  Allocates
+ * nothing and does not synchronise; work also runs on the handle's internal stream, ordered with
+ * `stream` by events, so synchronising `stream` is enough to observe the result. */
+mona_status mona_step(mona_handle* h, const mona_hparams* hp,
+                      void* const* params, const void* const* grads, void* stream);
+
+/* As mona_step, plus two measurement/verification hooks:
+ *   phase_mask : bit 0 prologue (lines 4-7, 10 + norm), bit 1 Newton-Schulz (line 8),
+ *                bit 2 parameter update (line 9).  7 = the full step.  A skipped phase leaves its
+ *                outputs as they were, so a partial mask is for timing only.
+ *   o_out      : NULL, or n_desc device pointers; descriptor i receives O_k in fp32 with the
+ *                parameter's own layout (rows x cols, batch_stride).  Entries may be NULL. */
+mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp,
+                         void* const* params, const void* const* grads, void* const* o_out,
+                         uint32_t phase_mask, void* stream);
+
+/* End-to-end variant for callers whose gradients arrive in HOST memory: for every descriptor copies
+ * grads_host[i] (pinned host memory, same layout and dtype as the device gradient, batch*batch_stride
+ * elements) into grads[i], runs the step, and copies the updated parameters back to params_host[i]
+ * (pinned, fp32).  Everything is enqueued on `stream`; nothing synchronises. */
+mona_status mona_step_host(mona_handle* h, const mona_hparams* hp,
+                           void* const* params, void* const* grads,
+                           const void* const* grads_host, void* const* params_host, void* stream);
+
+/* Synchronises `stream` and reads the device status word.  Returns MONA_OK, MONA_ERR_NONFINITE or
+ * MONA_ERR_TIMEOUT; *first_bad_matrix (may be NULL) receives the lowest global matrix index that
+ * reported a problem, or -1.  The word is cleared by the call. */
+mona_status mona_poll_status(mona_handle* h, void* stream, int64_t* first_bad_matrix);
+
+/* Byte offsets inside the state block of M, A and G_prev of matrix 0 of descriptor `desc`.  Matrix b
+ * of the descriptor follows at b * rows * cols * 4 bytes from each offset (state is stored densely,
+ * whatever batch_stride is).  A checkpoint is the state block plus the caller's own step count. */
+mona_status mona_state_layout(const mona_handle* h, int64_t desc,
+                              size_t* off_M, size_t* off_A, size_t* off_Gprev);
+
+/* Number of kernels the most recent mona_step*() call launched (for launch accounting). */
+int64_t mona_last_launch_count(const mona_handle* h);
+
+/* Counts of executed tensor-core work of the most recent step: bf16 multiply-add flops actually
+ * issued (2 * M * N * K summed over issued tile MMAs) and the dense-equivalent figure
+ * (4 s^2 l + 2 s^3 per matrix and iteration).  Either pointer may be NULL. */
+mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* dense_equivalent);
+
+/* Human-readable detail of the last failing call on this handle (never NULL). */
+const char* mona_last_error(const mona_handle* h);
+
+/* Frees the handle's tables, stream and events.  The caller's buffers are untouched. */
+void mona_destroy(mona_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MONA_H_ */

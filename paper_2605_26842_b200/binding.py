@@ -1,0 +1,200 @@
+"""ctypes binding of include/mona.h.  Names mirror the C entry points; nothing is computed here."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmona.so")
+
+STATUS_NAMES = {0: "MONA_OK", 1: "MONA_ERR_INVALID_ARG", 2: "MONA_ERR_UNSUPPORTED_SHAPE", 3: "MONA_ERR_ALIGNMENT",
+                4: "MONA_ERR_CUDA", 5: "MONA_ERR_TIMEOUT", 6: "MONA_ERR_NONFINITE", 7: "MONA_ERR_ARCH",
+                8: "MONA_ERR_BUFFER_TOO_SMALL"}
+MONA_F32, MONA_BF16 = 0, 1
+
+
+class MonaError(RuntimeError):
+    def __init__(self, status: int, detail: str = ""):
+        self.status = status
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {detail}")
+
+
+class MatrixDesc(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("batch", C.c_int64), ("batch_stride", C.c_int64),
+                ("grad_dtype", C.c_int32), ("reserved", C.c_int32)]
+
+
+class Hparams(C.Structure):
+    _fields_ = [("lr", C.c_double), ("momentum", C.c_double), ("accel_beta", C.c_double), ("accel_alpha", C.c_double),
+                ("weight_decay", C.c_double), ("ns_a", C.c_double), ("ns_b", C.c_double), ("ns_c", C.c_double),
+                ("norm_eps", C.c_double), ("scale_value", C.c_double), ("ns_steps", C.c_int32), ("scale_mode", C.c_int32),
+                ("ns_precision", C.c_int32), ("reserved", C.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libmona.so (once).  Raises if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2605_26842_b200.build` "
+                          "(needs nvcc; the library targets sm_100a and has no CPU fallback)")
+    L = C.CDLL(_LIB_PATH)
+    vp, vpp = C.c_void_p, C.POINTER(C.c_void_p)
+    L.mona_default_hparams.argtypes = [C.POINTER(Hparams)]
+    L.mona_set_chunk_budget.argtypes = [C.c_size_t]
+    L.mona_query_sizes.argtypes = [C.POINTER(MatrixDesc), C.c_int64, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.mona_create.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, vp, C.c_size_t, vp, C.c_size_t, C.c_int]
+    L.mona_step.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vp]
+    L.mona_step_ex.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, C.c_uint32, vp]
+    L.mona_step_host.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, vpp, vp]
+    L.mona_poll_status.argtypes = [vp, vp, C.POINTER(C.c_int64)]
+    L.mona_state_layout.argtypes = [vp, C.c_int64, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.mona_last_launch_count.argtypes = [vp]
+    L.mona_last_launch_count.restype = C.c_int64
+    L.mona_last_ns_flops.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    L.mona_last_error.argtypes = [vp]
+    L.mona_last_error.restype = C.c_char_p
+    L.mona_destroy.argtypes = [vp]
+    L.mona_destroy.restype = None
+    for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_query_sizes", "mona_create", "mona_step",
+                 "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops"):
+        getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def default_hparams(**overrides) -> Hparams:
+    hp = Hparams()
+    st = lib().mona_default_hparams(C.byref(hp))
+    if st:
+        raise MonaError(st)
+    for k, v in overrides.items():
+        if not hasattr(hp, k):
+            raise AttributeError(k)
+        setattr(hp, k, v)
+    return hp
+
+
+def set_chunk_budget(nbytes: int) -> None:
+    st = lib().mona_set_chunk_budget(nbytes)
+    if st:
+        raise MonaError(st, "chunk budget must be at least 1 MiB")
+
+
+def _desc_array(descs: Sequence[MatrixDesc]):
+    arr = (MatrixDesc * len(descs))()
+    for i, d in enumerate(descs):
+        arr[i] = d
+    return arr
+
+
+def query_sizes(descs: Sequence[MatrixDesc]):
+    sb, wb = C.c_size_t(0), C.c_size_t(0)
+    st = lib().mona_query_sizes(_desc_array(descs), len(descs), C.byref(sb), C.byref(wb))
+    if st:
+        raise MonaError(st, "mona_query_sizes")
+    return sb.value, wb.value
+
+
+def _ptr_array(tensors: Sequence[Optional[torch.Tensor]]):
+    arr = (C.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else t.data_ptr()
+    return arr
+
+
+class MonaOptimizer:
+    """Owns the state and workspace tensors (torch device memory) and a mona_handle.
+
+    `params[i]` is an fp32 CUDA tensor of shape (batch, rows, cols) or (rows, cols), contiguous;
+    `grads[i]` has the same shape in fp32 or bf16.  step() enqueues one optimizer step on the current
+    torch stream."""
+
+    def __init__(self, params: Sequence[torch.Tensor], grad_dtype=torch.float32, device: Optional[int] = None):
+        L = lib()
+        self.descs: List[MatrixDesc] = []
+        for p in params:
+            if p.dtype != torch.float32 or not p.is_contiguous() or p.dim() not in (2, 3):
+                raise ValueError("parameters must be contiguous fp32 tensors of shape (rows, cols) or (batch, rows, cols)")
+            batch = p.shape[0] if p.dim() == 3 else 1
+            rows, cols = p.shape[-2], p.shape[-1]
+            self.descs.append(MatrixDesc(rows, cols, batch, rows * cols, MONA_BF16 if grad_dtype == torch.bfloat16 else MONA_F32, 0))
+        self.device = torch.cuda.current_device() if device is None else device
+        self.grad_dtype = grad_dtype
+        sb, wb = query_sizes(self.descs)
+        dev = torch.device("cuda", self.device)
+        self.state = torch.empty(sb, dtype=torch.uint8, device=dev)
+        self.workspace = torch.empty(wb, dtype=torch.uint8, device=dev)
+        self._h = C.c_void_p()
+        st = L.mona_create(C.byref(self._h), _desc_array(self.descs), len(self.descs), self.state.data_ptr(), sb,
+                           self.workspace.data_ptr(), wb, self.device)
+        if st:
+            msg = L.mona_last_error(self._h).decode() if self._h else ""
+            L.mona_destroy(self._h)
+            self._h = None
+            raise MonaError(st, msg)
+
+    # -- helpers ---------------------------------------------------------------------------------
+    def _check(self, st: int):
+        if st:
+            raise MonaError(st, lib().mona_last_error(self._h).decode())
+
+    def _stream(self):
+        return C.c_void_p(torch.cuda.current_stream(self.device).cuda_stream)
+
+    # -- C entry points --------------------------------------------------------------------------
+    def step(self, hp: Hparams, params: Sequence[torch.Tensor], grads: Sequence[torch.Tensor]):
+        self._check(lib().mona_step(self._h, C.byref(hp), _ptr_array(params), _ptr_array(grads), self._stream()))
+
+    def step_ex(self, hp: Hparams, params, grads, o_out=None, phase_mask: int = 7):
+        o_arr = None if o_out is None else _ptr_array(o_out)
+        self._check(lib().mona_step_ex(self._h, C.byref(hp), _ptr_array(params), _ptr_array(grads), o_arr, phase_mask,
+                                       self._stream()))
+
+    def step_host(self, hp: Hparams, params, grads, grads_host, params_host):
+        self._check(lib().mona_step_host(self._h, C.byref(hp), _ptr_array(params), _ptr_array(grads),
+                                         _ptr_array(grads_host), _ptr_array(params_host), self._stream()))
+
+    def poll_status(self):
+        """Synchronises the current stream; returns (status code, first bad matrix index or -1)."""
+        bad = C.c_int64(-1)
+        st = lib().mona_poll_status(self._h, self._stream(), C.byref(bad))
+        return st, bad.value
+
+    def state_layout(self, desc: int):
+        a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+        self._check(lib().mona_state_layout(self._h, desc, C.byref(a), C.byref(b), C.byref(c)))
+        return a.value, b.value, c.value
+
+    def state_views(self, desc: int):
+        """fp32 views (batch, rows, cols) of M, A, G_prev of descriptor `desc` inside the state block."""
+        d = self.descs[desc]
+        n = d.batch * d.rows * d.cols
+        flat = self.state.view(torch.float32)
+        return tuple(flat[off // 4: off // 4 + n].view(d.batch, d.rows, d.cols) for off in self.state_layout(desc))
+
+    def last_launch_count(self) -> int:
+        return lib().mona_last_launch_count(self._h)
+
+    def last_ns_flops(self):
+        e, d = C.c_double(), C.c_double()
+        self._check(lib().mona_last_ns_flops(self._h, C.byref(e), C.byref(d)))
+        return e.value, d.value
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().mona_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,50 @@
+// Shared device-side declarations of the MONA step library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mona {
+
+// A chunk is the unit that goes through prologue -> Newton-Schulz -> update together: up to MAXC
+// same-shape matrices whose bf16 iterates fit the L2 budget.
+constexpr int MAXC = 64;
+// Each matrix is cut into at most MAX_SLABS contiguous slabs for the elementwise passes; every slab
+// owns one partial sum of squares, so the Frobenius norm is reduced in a fixed order.
+constexpr int MAX_SLABS = 256;
+
+// Per-chunk pointer table passed by value to the elementwise kernels.
+struct ChunkPtrs {
+    const void* g[MAXC];   // gradient of matrix c (fp32 or bf16)
+    float* w[MAXC];        // parameter of matrix c
+    float* o[MAXC];        // optional fp32 copy of O_k (may be null)
+    int gid[MAXC];         // global matrix index (descriptor order), for error reports
+};
+
+// Device status word, latched by kernels and read by mona_poll_status().
+struct DeviceStatus {
+    unsigned int flags;        // bit 0: non-finite norm, bit 1: a bounded wait ran out
+    int first_bad;             // lowest global matrix index that reported (or INT_MAX)
+    unsigned int timeout_site; // which wait gave up (diagnostic)
+    unsigned int pad;
+};
+constexpr unsigned STATUS_NONFINITE = 1u;
+constexpr unsigned STATUS_TIMEOUT = 2u;
+
+// A scalar hyper-parameter carried as an unevaluated sum of two floats, hi + lo, so that products with
+// it are accurate to ~2^-45 instead of 2^-24: rounding beta_a = 0.99 to one float would by itself
+// cost 3e-8 per step in the EMA, which accumulates over its ~1/(1-beta_a) step memory.
+struct F2 {
+    float hi, lo;
+};
+
+struct PrologueScalars {
+    F2 beta;            // beta_a
+    F2 one_minus_beta;  // 1 - beta_a, formed in double
+    F2 alpha;           // alpha
+    F2 mu;              // mu
+    float eps;          // norm_eps
+};
+
+}  // namespace mona

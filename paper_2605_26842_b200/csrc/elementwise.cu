@@ -1,0 +1,240 @@
+// Elementwise passes of the MONA step: the fused prologue (Algorithm 1 lines 4-7 and 10 plus the
+// Frobenius norm that Eq. newton_schulz starts from) and the parameter update (line 9).
+// Both are single HBM passes over contiguous slabs with 128-bit accesses.
+#include "elementwise.cuh"
+
+#include <math.h>
+
+namespace mona {
+
+namespace {
+
+constexpr int EW_THREADS = 256;
+
+__device__ __forceinline__ float mul_add2(F2 k, float x, float addend) {
+    // (k.hi + k.lo) * x + addend with a single rounding on the dominant term
+    return fmaf(k.hi, x, fmaf(k.lo, x, addend));
+}
+
+template <typename GT>
+struct GradLoad;
+template <>
+struct GradLoad<float> {
+    static __device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ float load1(const float* p) { return __ldcs(p); }
+};
+template <>
+struct GradLoad<__nv_bfloat16> {
+    static __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+        uint2 raw = __ldcs(reinterpret_cast<const uint2*>(p));
+        float4 r;
+        r.x = __uint_as_float(raw.x << 16);
+        r.y = __uint_as_float(raw.x & 0xffff0000u);
+        r.z = __uint_as_float(raw.y << 16);
+        r.w = __uint_as_float(raw.y & 0xffff0000u);
+        return r;
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+};
+
+__device__ __forceinline__ void mona_elem(float g, float& gp, float& a, float& m, const PrologueScalars& k) {
+    float d = g - gp;                                              // D_k = G_k - G_{k-1}
+    a = mul_add2(k.beta, a, fmaf(k.one_minus_beta.hi, d, k.one_minus_beta.lo * d));  // A_k
+    float gt = mul_add2(k.alpha, a, g);                             // G~_k = G_k + alpha A_k
+    m = mul_add2(k.mu, m, gt);                                      // M_k = mu M_{k-1} + G~_k
+    gp = g;                                                         // G_{k-1} <- G_k
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float block_sum(float v, float* smem /* >= 8 floats */) {
+    #pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) smem[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (warp == 0) {
+        t = (lane < (EW_THREADS >> 5)) ? smem[lane] : 0.f;
+        #pragma unroll
+        for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    }
+    return t;   // valid in warp 0 (all lanes)
+}
+
+// grid = (slabs, C).  Block (p, c) owns elements [p*slab_len, min(e, (p+1)*slab_len)) of matrix c.
+// The last block of a matrix to finish adds the slab partials in index order, so ||M||_F does not
+// depend on scheduling; it then resets the arrival counter for the next call.
+template <typename GT, int VEC>
+__global__ void __launch_bounds__(EW_THREADS)
+prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, float* __restrict__ Ast, float* __restrict__ Gpst,
+                __nv_bfloat16* __restrict__ xhat, float* __restrict__ partials, unsigned int* __restrict__ counters,
+                float* __restrict__ inv_norm, DeviceStatus* __restrict__ status, long long e, long long slab_len,
+                int slabs, PrologueScalars k) {
+    __shared__ float red[8];
+    __shared__ int is_last;
+    const int c = blockIdx.y, p = blockIdx.x;
+    const long long lo = (long long)p * slab_len;
+    const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
+    const GT* __restrict__ g = reinterpret_cast<const GT*>(ptrs.g[c]);
+    float* __restrict__ M = Mst + (long long)c * e;
+    float* __restrict__ A = Ast + (long long)c * e;
+    float* __restrict__ Gp = Gpst + (long long)c * e;
+    __nv_bfloat16* __restrict__ X = xhat ? xhat + (long long)c * e : nullptr;
+
+    float acc = 0.f;
+    if (VEC == 4) {
+        constexpr long long STEP = (long long)EW_THREADS * 4;
+        long long i = lo + (long long)threadIdx.x * 4;
+        // two independent vectors per trip keep ~128 B per thread in flight
+        for (; i + STEP < hi; i += 2 * STEP) {
+            float4 g0 = GradLoad<GT>::load4(g + i), g1 = GradLoad<GT>::load4(g + i + STEP);
+            float4 p0 = __ldcs(reinterpret_cast<const float4*>(Gp + i)), p1 = __ldcs(reinterpret_cast<const float4*>(Gp + i + STEP));
+            float4 a0 = __ldcs(reinterpret_cast<const float4*>(A + i)), a1 = __ldcs(reinterpret_cast<const float4*>(A + i + STEP));
+            float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i)), m1 = __ldcs(reinterpret_cast<const float4*>(M + i + STEP));
+            mona_elem(g0.x, p0.x, a0.x, m0.x, k); mona_elem(g0.y, p0.y, a0.y, m0.y, k);
+            mona_elem(g0.z, p0.z, a0.z, m0.z, k); mona_elem(g0.w, p0.w, a0.w, m0.w, k);
+            mona_elem(g1.x, p1.x, a1.x, m1.x, k); mona_elem(g1.y, p1.y, a1.y, m1.y, k);
+            mona_elem(g1.z, p1.z, a1.z, m1.z, k); mona_elem(g1.w, p1.w, a1.w, m1.w, k);
+            __stcs(reinterpret_cast<float4*>(Gp + i), p0); __stcs(reinterpret_cast<float4*>(Gp + i + STEP), p1);
+            __stcs(reinterpret_cast<float4*>(A + i), a0);  __stcs(reinterpret_cast<float4*>(A + i + STEP), a1);
+            __stcs(reinterpret_cast<float4*>(M + i), m0);  __stcs(reinterpret_cast<float4*>(M + i + STEP), m1);
+            if (X) {
+                *reinterpret_cast<uint2*>(X + i) = make_uint2(pack_bf16x2(m0.x, m0.y), pack_bf16x2(m0.z, m0.w));
+                *reinterpret_cast<uint2*>(X + i + STEP) = make_uint2(pack_bf16x2(m1.x, m1.y), pack_bf16x2(m1.z, m1.w));
+            }
+            acc = fmaf(m0.x, m0.x, acc); acc = fmaf(m0.y, m0.y, acc); acc = fmaf(m0.z, m0.z, acc); acc = fmaf(m0.w, m0.w, acc);
+            acc = fmaf(m1.x, m1.x, acc); acc = fmaf(m1.y, m1.y, acc); acc = fmaf(m1.z, m1.z, acc); acc = fmaf(m1.w, m1.w, acc);
+        }
+        for (; i < hi; i += STEP) {
+            float4 g0 = GradLoad<GT>::load4(g + i);
+            float4 p0 = __ldcs(reinterpret_cast<const float4*>(Gp + i));
+            float4 a0 = __ldcs(reinterpret_cast<const float4*>(A + i));
+            float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i));
+            mona_elem(g0.x, p0.x, a0.x, m0.x, k); mona_elem(g0.y, p0.y, a0.y, m0.y, k);
+            mona_elem(g0.z, p0.z, a0.z, m0.z, k); mona_elem(g0.w, p0.w, a0.w, m0.w, k);
+            __stcs(reinterpret_cast<float4*>(Gp + i), p0);
+            __stcs(reinterpret_cast<float4*>(A + i), a0);
+            __stcs(reinterpret_cast<float4*>(M + i), m0);
+            if (X) *reinterpret_cast<uint2*>(X + i) = make_uint2(pack_bf16x2(m0.x, m0.y), pack_bf16x2(m0.z, m0.w));
+            acc = fmaf(m0.x, m0.x, acc); acc = fmaf(m0.y, m0.y, acc); acc = fmaf(m0.z, m0.z, acc); acc = fmaf(m0.w, m0.w, acc);
+        }
+    } else {
+        for (long long i = lo + threadIdx.x; i < hi; i += EW_THREADS) {
+            float gv = GradLoad<GT>::load1(g + i), pv = Gp[i], av = A[i], mv = M[i];
+            mona_elem(gv, pv, av, mv, k);
+            Gp[i] = pv; A[i] = av; M[i] = mv;
+            if (X) X[i] = __float2bfloat16_rn(mv);
+            acc = fmaf(mv, mv, acc);
+        }
+    }
+
+    float total = block_sum(acc, red);
+    if (threadIdx.x == 0) {
+        __stcg(partials + (long long)c * MAX_SLABS + p, total);
+        __threadfence();
+        unsigned int prev = atomicAdd(counters + c, 1u);
+        is_last = (prev == (unsigned int)(slabs - 1));
+    }
+    __syncthreads();
+    if (is_last && threadIdx.x < 32) {
+        __threadfence();
+        double s = 0.0;
+        for (int j = threadIdx.x; j < slabs; j += 32) s += (double)__ldcg(partials + (long long)c * MAX_SLABS + j);
+        #pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (threadIdx.x == 0) {
+            float nrm = (float)sqrt(s);
+            inv_norm[c] = 1.0f / (nrm + k.eps);        // X_0 = M / (||M||_F + eps)
+            if (!isfinite(nrm)) {
+                atomicOr(&status->flags, STATUS_NONFINITE);
+                atomicMin(&status->first_bad, ptrs.gid[c]);
+            }
+            counters[c] = 0u;
+        }
+    }
+}
+
+// W <- W - eta (gamma O + lambda W), evaluated as (W - (eta lambda) W) - (eta gamma) O.
+template <typename OT, int VEC>
+__global__ void __launch_bounds__(EW_THREADS)
+update_kernel(ChunkPtrs ptrs, const OT* __restrict__ O, long long e, long long slab_len, float eta_lambda,
+              float eta_gamma) {
+    const int c = blockIdx.y, p = blockIdx.x;
+    const long long lo = (long long)p * slab_len;
+    const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
+    float* __restrict__ W = ptrs.w[c];
+    float* __restrict__ Oout = ptrs.o[c];
+    const OT* __restrict__ Oc = O + (long long)c * e;
+    if (VEC == 4) {
+        for (long long i = lo + (long long)threadIdx.x * 4; i < hi; i += (long long)EW_THREADS * 4) {
+            float4 w = __ldcs(reinterpret_cast<const float4*>(W + i));
+            float4 o = GradLoad<OT>::load4(Oc + i);
+            w.x = fmaf(-eta_gamma, o.x, fmaf(-eta_lambda, w.x, w.x));
+            w.y = fmaf(-eta_gamma, o.y, fmaf(-eta_lambda, w.y, w.y));
+            w.z = fmaf(-eta_gamma, o.z, fmaf(-eta_lambda, w.z, w.z));
+            w.w = fmaf(-eta_gamma, o.w, fmaf(-eta_lambda, w.w, w.w));
+            __stcs(reinterpret_cast<float4*>(W + i), w);
+            if (Oout) *reinterpret_cast<float4*>(Oout + i) = o;
+        }
+    } else {
+        for (long long i = lo + threadIdx.x; i < hi; i += EW_THREADS) {
+            float w = W[i], o = GradLoad<OT>::load1(Oc + i);
+            W[i] = fmaf(-eta_gamma, o, fmaf(-eta_lambda, w, w));
+            if (Oout) Oout[i] = o;
+        }
+    }
+}
+
+// X_0 = M * inv_norm (fp32 validation path only).
+__global__ void __launch_bounds__(EW_THREADS)
+scale_kernel(const float* __restrict__ M, float* __restrict__ X, const float* __restrict__ inv_norm, long long e,
+             long long slab_len) {
+    const int c = blockIdx.y;
+    const long long lo = (long long)blockIdx.x * slab_len;
+    const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
+    const float s = inv_norm[c];
+    for (long long i = lo + threadIdx.x; i < hi; i += EW_THREADS) X[(long long)c * e + i] = M[(long long)c * e + i] * s;
+}
+
+}  // namespace
+
+cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool vec4, float* M, float* A, float* Gp,
+                            __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm,
+                            DeviceStatus* status, long long e, long long slab_len, int slabs,
+                            const PrologueScalars& k, cudaStream_t stream) {
+    dim3 grid(slabs, C), block(EW_THREADS);
+    if (grad_bf16) {
+        if (vec4) prologue_kernel<__nv_bfloat16, 4><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        else      prologue_kernel<__nv_bfloat16, 1><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+    } else {
+        if (vec4) prologue_kernel<float, 4><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        else      prologue_kernel<float, 1><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_update(const ChunkPtrs& ptrs, int C, bool o_is_bf16, bool vec4, const void* O, long long e,
+                          long long slab_len, int slabs, float eta_lambda, float eta_gamma, cudaStream_t stream) {
+    dim3 grid(slabs, C), block(EW_THREADS);
+    if (o_is_bf16) {
+        if (vec4) update_kernel<__nv_bfloat16, 4><<<grid, block, 0, stream>>>(ptrs, (const __nv_bfloat16*)O, e, slab_len, eta_lambda, eta_gamma);
+        else      update_kernel<__nv_bfloat16, 1><<<grid, block, 0, stream>>>(ptrs, (const __nv_bfloat16*)O, e, slab_len, eta_lambda, eta_gamma);
+    } else {
+        if (vec4) update_kernel<float, 4><<<grid, block, 0, stream>>>(ptrs, (const float*)O, e, slab_len, eta_lambda, eta_gamma);
+        else      update_kernel<float, 1><<<grid, block, 0, stream>>>(ptrs, (const float*)O, e, slab_len, eta_lambda, eta_gamma);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale(const float* M, float* X, const float* inv_norm, int C, long long e, long long slab_len,
+                         int slabs, cudaStream_t stream) {
+    dim3 grid(slabs, C), block(EW_THREADS);
+    scale_kernel<<<grid, block, 0, stream>>>(M, X, inv_norm, e, slab_len);
+    return cudaGetLastError();
+}
+
+}  // namespace mona

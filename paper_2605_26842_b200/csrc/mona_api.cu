@@ -1,0 +1,499 @@
+// C ABI of the MONA step library: plan (shape buckets, chunking, state/workspace layout, TMA descriptors)
+// and the per-step launch sequence.  See include/mona.h for the contract of every entry point.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <climits>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/mona.h"
+#include "common.cuh"
+#include "elementwise.cuh"
+#include "ns_fp32.cuh"
+#include "ns_tc.cuh"
+
+using namespace mona;
+
+namespace {
+
+// ---- workspace layout -------------------------------------------------------------------------------
+constexpr size_t WS_STATUS_OFF = 0;
+constexpr size_t WS_COUNTERS_OFF = 256;
+constexpr size_t WS_INVNORM_OFF = 1024;
+constexpr size_t WS_PARTIALS_OFF = 4096;
+constexpr size_t WS_DATA_OFF = 128 * 1024;
+static_assert(WS_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS <= WS_DATA_OFF, "control block overflow");
+
+// Bytes of bf16 iterates (X_t, X_{t+1}, A_t, B_t) a chunk may hold so that it stays resident in L2
+// between the 3T GEMMs of the iteration.
+size_t g_chunk_budget_bytes = 48ull << 20;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct MatRef {
+    int desc;
+    int64_t b;
+};
+
+struct Bucket {
+    int64_t rows = 0, cols = 0, s = 0, l = 0, e = 0;
+    int grad_dtype = 0;
+    bool tall = false, tc_ok = false;
+    std::vector<MatRef> mats;
+    int64_t state_off = 0;      // floats from the state base: M block, then A block, then G_prev block
+    int Cb = 1, Cf = 1;         // chunk capacity: bf16 tensor-core mode / fp32 mode
+    int slabs = 1;
+    int64_t slab_len = 0;
+    size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;          // bf16 mode, bytes from workspace base
+    size_t off32_x[2] = {0, 0}, off32_a = 0, off32_b = 0;    // fp32 mode
+    size_t data_bytes = 0;
+    CUtensorMap tm_x[2], tm_a, tm_b;
+};
+
+struct Plan {
+    std::vector<mona_matrix_desc> descs;
+    std::vector<Bucket> buckets;
+    std::vector<int> desc_bucket;          // bucket of descriptor i
+    std::vector<int64_t> desc_pos;         // position of descriptor i's matrix 0 inside its bucket
+    std::vector<int64_t> desc_first_gid;   // global matrix index (descriptor order) of matrix 0
+    size_t state_bytes = 0, workspace_bytes = 0;
+};
+
+mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan, std::string& err) {
+    if (!descs || n_desc <= 0) { err = "descs is null or n_desc <= 0"; return MONA_ERR_INVALID_ARG; }
+    plan.descs.assign(descs, descs + n_desc);
+    std::map<std::tuple<int64_t, int64_t, int>, int> index;
+    int64_t gid = 0;
+    for (int64_t i = 0; i < n_desc; ++i) {
+        mona_matrix_desc& d = plan.descs[i];
+        if (d.rows <= 0 || d.cols <= 0 || d.batch <= 0) { err = "descriptor with non-positive rows/cols/batch"; return MONA_ERR_INVALID_ARG; }
+        if (d.grad_dtype != MONA_F32 && d.grad_dtype != MONA_BF16) { err = "descriptor with unknown grad_dtype"; return MONA_ERR_INVALID_ARG; }
+        if (d.rows > (1 << 20) || d.cols > (1 << 20) || d.rows * d.cols > (1ll << 31)) { err = "matrix too large"; return MONA_ERR_UNSUPPORTED_SHAPE; }
+        if (d.batch_stride == 0) d.batch_stride = d.rows * d.cols;
+        if (d.batch_stride < d.rows * d.cols) { err = "batch_stride smaller than rows*cols"; return MONA_ERR_INVALID_ARG; }
+        auto key = std::make_tuple(d.rows, d.cols, (int)d.grad_dtype);
+        auto it = index.find(key);
+        int bi;
+        if (it == index.end()) {
+            bi = (int)plan.buckets.size();
+            index[key] = bi;
+            Bucket b;
+            b.rows = d.rows; b.cols = d.cols; b.grad_dtype = d.grad_dtype;
+            b.tall = d.rows > d.cols;
+            b.s = std::min(d.rows, d.cols); b.l = std::max(d.rows, d.cols); b.e = d.rows * d.cols;
+            b.tc_ok = (b.s % 8 == 0) && (b.l % 8 == 0) && b.s >= 64;
+            plan.buckets.push_back(b);
+        } else {
+            bi = it->second;
+        }
+        plan.desc_bucket.push_back(bi);
+        plan.desc_pos.push_back((int64_t)plan.buckets[bi].mats.size());
+        plan.desc_first_gid.push_back(gid);
+        for (int64_t b = 0; b < d.batch; ++b) plan.buckets[bi].mats.push_back({(int)i, b});
+        gid += d.batch;
+    }
+    int64_t state_floats = 0;
+    size_t max_data = 0;
+    for (Bucket& b : plan.buckets) {
+        const int64_t count = (int64_t)b.mats.size();
+        b.state_off = state_floats;
+        state_floats += 3 * count * b.e;
+        state_floats = (int64_t)align_up((size_t)state_floats, 64);        // keep every block 256-byte aligned
+        // slabs: ~16K elements each, at most MAX_SLABS, slab length a multiple of 1024
+        int64_t slab = 16384;
+        if ((b.e + slab - 1) / slab > MAX_SLABS) slab = (int64_t)align_up((size_t)((b.e + MAX_SLABS - 1) / MAX_SLABS), 1024);
+        b.slab_len = slab;
+        b.slabs = (int)((b.e + slab - 1) / slab);
+        // chunk capacity
+        const size_t per_mat_bf16 = (size_t)(2 * b.e + 2 * b.s * b.s) * 2;
+        int64_t cb = (int64_t)(g_chunk_budget_bytes / per_mat_bf16);
+        cb = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(cb, MAXC), count));
+        b.Cb = (int)cb;
+        b.Cf = (int)std::max<int64_t>(1, cb / 2);
+        size_t off = WS_DATA_OFF;
+        for (int i = 0; i < 2; ++i) { b.off_x[i] = off; off += align_up((size_t)b.Cb * b.e * 2, 1024); }
+        b.off_a = off; off += align_up((size_t)b.Cb * b.s * b.s * 2, 1024);
+        b.off_b = off; off += align_up((size_t)b.Cb * b.s * b.s * 2, 1024);
+        size_t off32 = WS_DATA_OFF;
+        for (int i = 0; i < 2; ++i) { b.off32_x[i] = off32; off32 += align_up((size_t)b.Cf * b.e * 4, 1024); }
+        b.off32_a = off32; off32 += align_up((size_t)b.Cf * b.s * b.s * 4, 1024);
+        b.off32_b = off32; off32 += align_up((size_t)b.Cf * b.s * b.s * 4, 1024);
+        b.data_bytes = std::max(off, off32);
+        max_data = std::max(max_data, b.data_bytes);
+    }
+    plan.state_bytes = (size_t)state_floats * 4;
+    plan.workspace_bytes = max_data;
+    return MONA_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 tensor [C][outer][inner] (inner contiguous) cut into 64 x 64 boxes with the 128-byte swizzle.
+bool encode_map(EncodeTiledFn fn, CUtensorMap* map, void* base, int64_t inner, int64_t outer, int64_t C) {
+    cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)C};
+    cuuint64_t strides[2] = {(cuuint64_t)inner * 2, (cuuint64_t)inner * (cuuint64_t)outer * 2};
+    cuuint32_t box[3] = {(cuuint32_t)TC_BOX, (cuuint32_t)TC_BOX, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+F2 split(double v) {
+    F2 r;
+    r.hi = (float)v;
+    r.lo = (float)(v - (double)r.hi);
+    return r;
+}
+
+}  // namespace
+
+struct mona_handle {
+    Plan plan;
+    int device = 0, num_sms = 0;
+    uint8_t* state = nullptr;
+    uint8_t* ws = nullptr;
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    DeviceStatus* host_status = nullptr;   // pinned
+    std::string last_error;
+    int64_t launches = 0;
+    double flops_exec = 0.0, flops_dense = 0.0;
+
+    mona_status fail(mona_status st, const char* fmt, ...) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        last_error = buf;
+        return st;
+    }
+};
+
+#define MONA_CUDA(h, call)                                                                                 \
+    do {                                                                                                   \
+        cudaError_t e_ = (call);                                                                           \
+        if (e_ != cudaSuccess) return (h)->fail(MONA_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+extern "C" {
+
+mona_status mona_default_hparams(mona_hparams* hp) {
+    if (!hp) return MONA_ERR_INVALID_ARG;
+    memset(hp, 0, sizeof *hp);
+    hp->lr = 1e-3; hp->momentum = 0.95; hp->accel_beta = 0.99; hp->accel_alpha = -1.0 / (2.0 * (1.0 - 0.99));
+    hp->weight_decay = 0.1; hp->ns_a = 3.4445; hp->ns_b = -4.7750; hp->ns_c = 2.0315; hp->norm_eps = 1e-7;
+    hp->scale_value = 0.2; hp->ns_steps = 5; hp->scale_mode = 0; hp->ns_precision = 0;
+    return MONA_OK;
+}
+
+mona_status mona_set_chunk_budget(size_t bytes) {
+    if (bytes < (1u << 20)) return MONA_ERR_INVALID_ARG;
+    g_chunk_budget_bytes = bytes;
+    return MONA_OK;
+}
+
+mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc, size_t* state_bytes, size_t* workspace_bytes) {
+    Plan plan;
+    std::string err;
+    mona_status st = build_plan(descs, n_desc, plan, err);
+    if (st != MONA_OK) return st;
+    if (state_bytes) *state_bytes = plan.state_bytes;
+    if (workspace_bytes) *workspace_bytes = plan.workspace_bytes;
+    return MONA_OK;
+}
+
+mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc, void* state, size_t state_bytes,
+                        void* workspace, size_t workspace_bytes, int device) {
+    if (!out) return MONA_ERR_INVALID_ARG;
+    *out = nullptr;
+    mona_handle* h = new mona_handle();
+    *out = h;     // returned even on failure so that mona_last_error() can be read; destroy it either way
+    mona_status st = build_plan(descs, n_desc, h->plan, h->last_error);
+    if (st != MONA_OK) return st;
+    if (!state || !workspace) return h->fail(MONA_ERR_INVALID_ARG, "state or workspace is null");
+    if (((uintptr_t)state & 255) || ((uintptr_t)workspace & 255)) return h->fail(MONA_ERR_ALIGNMENT, "state/workspace must be 256-byte aligned");
+    if (state_bytes < h->plan.state_bytes || workspace_bytes < h->plan.workspace_bytes)
+        return h->fail(MONA_ERR_BUFFER_TOO_SMALL, "need state %zu B, workspace %zu B", h->plan.state_bytes, h->plan.workspace_bytes);
+    int ndev = 0;
+    cudaError_t ce = cudaGetDeviceCount(&ndev);
+    if (ce != cudaSuccess || device < 0 || device >= ndev)
+        return h->fail(MONA_ERR_CUDA, "no usable CUDA device %d (%s)", device, cudaGetErrorString(ce));
+    MONA_CUDA(h, cudaSetDevice(device));
+    cudaDeviceProp prop;
+    MONA_CUDA(h, cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return h->fail(MONA_ERR_ARCH, "device %d is sm_%d%d; this library is built for sm_100a only", device, prop.major, prop.minor);
+    h->device = device;
+    h->num_sms = prop.multiProcessorCount;
+    h->state = (uint8_t*)state;
+    h->ws = (uint8_t*)workspace;
+
+    EncodeTiledFn encode = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    MONA_CUDA(h, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", (void**)&encode, cudaEnableDefault, &qres));
+    if (!encode || qres != cudaDriverEntryPointSuccess) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled not available");
+    for (Bucket& b : h->plan.buckets) {
+        if (!b.tc_ok) continue;
+        bool ok = true;
+        for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.tm_x[i], h->ws + b.off_x[i], b.cols, b.rows, b.Cb);
+        ok = ok && encode_map(encode, &b.tm_a, h->ws + b.off_a, b.s, b.s, b.Cb);
+        ok = ok && encode_map(encode, &b.tm_b, h->ws + b.off_b, b.s, b.s, b.Cb);
+        if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
+    }
+    MONA_CUDA(h, tc_gemm_configure());
+    MONA_CUDA(h, cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
+    MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
+    MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
+    MONA_CUDA(h, cudaMallocHost((void**)&h->host_status, sizeof(DeviceStatus)));
+    // M_0 = A_0 = G_0 = 0; control block cleared
+    MONA_CUDA(h, cudaMemset(h->state, 0, h->plan.state_bytes));
+    MONA_CUDA(h, cudaMemset(h->ws, 0, WS_DATA_OFF));
+    DeviceStatus init = {0u, INT_MAX, 0u, 0u};
+    MONA_CUDA(h, cudaMemcpy(h->ws + WS_STATUS_OFF, &init, sizeof init, cudaMemcpyHostToDevice));
+    MONA_CUDA(h, cudaDeviceSynchronize());
+    return MONA_OK;
+}
+
+mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads,
+                         void* const* o_out, uint32_t phase_mask, void* stream_v) {
+    if (!h) return MONA_ERR_INVALID_ARG;
+    if (!hp || !params || !grads) return h->fail(MONA_ERR_INVALID_ARG, "hp, params or grads is null");
+    if (hp->ns_steps < 0 || hp->ns_steps > 64) return h->fail(MONA_ERR_INVALID_ARG, "ns_steps out of range");
+    if (hp->ns_precision != 0 && hp->ns_precision != 1) return h->fail(MONA_ERR_INVALID_ARG, "ns_precision must be 0 or 1");
+    if (hp->scale_mode != 0 && hp->scale_mode != 1) return h->fail(MONA_ERR_INVALID_ARG, "scale_mode must be 0 or 1");
+    const Plan& plan = h->plan;
+    const int64_t n_desc = (int64_t)plan.descs.size();
+    for (int64_t i = 0; i < n_desc; ++i) {
+        if (!params[i] || !grads[i]) return h->fail(MONA_ERR_INVALID_ARG, "params[%lld] or grads[%lld] is null", (long long)i, (long long)i);
+        if (((uintptr_t)params[i] & 15) || ((uintptr_t)grads[i] & 15) || (o_out && o_out[i] && ((uintptr_t)o_out[i] & 15)))
+            return h->fail(MONA_ERR_ALIGNMENT, "descriptor %lld: pointers must be 16-byte aligned", (long long)i);
+    }
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    MONA_CUDA(h, cudaSetDevice(h->device));
+
+    PrologueScalars ps;
+    ps.beta = split(hp->accel_beta);
+    ps.one_minus_beta = split(1.0 - hp->accel_beta);
+    ps.alpha = split(hp->accel_alpha);
+    ps.mu = split(hp->momentum);
+    ps.eps = (float)hp->norm_eps;
+    const float eta_lambda = (float)(hp->lr * hp->weight_decay);
+    const int T = hp->ns_steps;
+    const float ns_a = (float)hp->ns_a, ns_b = (float)hp->ns_b, ns_c = (float)hp->ns_c;
+
+    DeviceStatus* dstatus = (DeviceStatus*)(h->ws + WS_STATUS_OFF);
+    unsigned int* counters = (unsigned int*)(h->ws + WS_COUNTERS_OFF);
+    float* inv_norm = (float*)(h->ws + WS_INVNORM_OFF);
+    float* partials = (float*)(h->ws + WS_PARTIALS_OFF);
+    h->launches = 0;
+    h->flops_exec = 0.0;
+    h->flops_dense = 0.0;
+
+    for (const Bucket& b : plan.buckets) {
+        const bool tc = (hp->ns_precision == 0) && b.tc_ok && T >= 1;
+        const int cap = tc ? b.Cb : b.Cf;
+        const int64_t count = (int64_t)b.mats.size();
+        const double gamma = hp->scale_mode == 0 ? hp->scale_value * std::sqrt((double)b.l) : hp->scale_value;
+        const float eta_gamma = (float)(hp->lr * gamma);
+        float* Mst = (float*)h->state + b.state_off;
+        float* Ast = Mst + count * b.e;
+        float* Gst = Ast + count * b.e;
+        const size_t gsz = b.grad_dtype == MONA_BF16 ? 2 : 4;
+
+        for (int64_t start = 0; start < count; start += cap) {
+            const int C = (int)std::min<int64_t>(cap, count - start);
+            ChunkPtrs ptrs;
+            bool vec4 = (b.e % 4 == 0);
+            for (int c = 0; c < C; ++c) {
+                const MatRef& mr = b.mats[start + c];
+                const mona_matrix_desc& d = plan.descs[mr.desc];
+                if ((d.batch_stride * (int64_t)gsz) % 16 != 0 || (d.batch_stride * 4) % 16 != 0) vec4 = false;
+                ptrs.g[c] = (const uint8_t*)grads[mr.desc] + (size_t)mr.b * d.batch_stride * gsz;
+                ptrs.w[c] = (float*)params[mr.desc] + mr.b * d.batch_stride;
+                ptrs.o[c] = (o_out && o_out[mr.desc]) ? (float*)o_out[mr.desc] + mr.b * d.batch_stride : nullptr;
+                ptrs.gid[c] = (int)(plan.desc_first_gid[mr.desc] + mr.b);
+            }
+            float* Mc = Mst + start * b.e;
+            float* Ac = Ast + start * b.e;
+            float* Gc = Gst + start * b.e;
+            __nv_bfloat16* xb[2] = {(__nv_bfloat16*)(h->ws + b.off_x[0]), (__nv_bfloat16*)(h->ws + b.off_x[1])};
+            __nv_bfloat16* ab = (__nv_bfloat16*)(h->ws + b.off_a);
+            __nv_bfloat16* bb = (__nv_bfloat16*)(h->ws + b.off_b);
+            float* xf[2] = {(float*)(h->ws + b.off32_x[0]), (float*)(h->ws + b.off32_x[1])};
+            float* af = (float*)(h->ws + b.off32_a);
+            float* bf = (float*)(h->ws + b.off32_b);
+
+            if (phase_mask & 1u) {
+                MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16, vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
+                                             counters, inv_norm, dstatus, b.e, b.slab_len, b.slabs, ps, stream));
+                ++h->launches;
+            }
+            const void* o_final = nullptr;
+            if (tc) {
+                if (phase_mask & 2u) {
+                    for (int t = 0; t < T; ++t) {
+                        const int cur = t & 1, nxt = cur ^ 1;
+                        TcGemm g1{};
+                        g1.C = C; g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_mn = g1.b_mn = b.tall ? 1 : 0; g1.symmetric = 1;
+                        g1.cin = nullptr; g1.out = ab; g1.ld = b.s; g1.mat_stride = b.s * b.s; g1.c1 = 0.f; g1.c2 = 1.f;
+                        g1.inv_norm = inv_norm; g1.post_mode = t == 0 ? 2 : 0;
+                        tc_gemm_plan(g1);
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_x[cur], g1, h->num_sms, dstatus, stream));
+                        TcGemm g2{};
+                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_mn = g2.b_mn = 0; g2.symmetric = 1;
+                        g2.cin = ab; g2.out = bb; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
+                        g2.inv_norm = inv_norm; g2.post_mode = 0;
+                        tc_gemm_plan(g2);
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_a, b.tm_a, g2, h->num_sms, dstatus, stream));
+                        TcGemm g3{};
+                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0;
+                        g3.cin = xb[cur]; g3.out = xb[nxt]; g3.ld = b.cols; g3.mat_stride = b.e; g3.c1 = ns_a; g3.c2 = 1.f;
+                        g3.inv_norm = inv_norm; g3.post_mode = t == 0 ? 1 : 0;
+                        if (!b.tall) {   // X' = a X + B X : B is the K-major "A" operand, X the MN-major "B" operand
+                            g3.M = (int)b.s; g3.N = (int)b.l; g3.a_mn = 0; g3.b_mn = 1;
+                            tc_gemm_plan(g3);
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_b, b.tm_x[cur], g3, h->num_sms, dstatus, stream));
+                        } else {         // X' = a X + X B : X is K-major, B (symmetric) serves as its own transpose
+                            g3.M = (int)b.l; g3.N = (int)b.s; g3.a_mn = 0; g3.b_mn = 0;
+                            tc_gemm_plan(g3);
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_b, g3, h->num_sms, dstatus, stream));
+                        }
+                        h->launches += 3;
+                        h->flops_exec += tc_gemm_executed_flops(g1) + tc_gemm_executed_flops(g2) + tc_gemm_executed_flops(g3);
+                        h->flops_dense += (double)C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
+                    }
+                }
+                o_final = xb[T & 1];
+            } else {
+                if (phase_mask & 2u) {
+                    MONA_CUDA(h, launch_scale(Mc, xf[0], inv_norm, C, b.e, b.slab_len, b.slabs, stream));
+                    ++h->launches;
+                    for (int t = 0; t < T; ++t) {
+                        const int cur = t & 1, nxt = cur ^ 1;
+                        SgemmArgs g1{};   // A = X X^T (wide) or X^T X (tall), s x s
+                        g1.a = xf[cur]; g1.b = xf[cur]; g1.a_batch = g1.b_batch = b.e;
+                        if (!b.tall) { g1.a_si = b.cols; g1.a_sk = 1; g1.b_sk = 1; g1.b_sj = b.cols; }
+                        else         { g1.a_si = 1; g1.a_sk = b.cols; g1.b_sk = b.cols; g1.b_sj = 1; }
+                        g1.cin = nullptr; g1.d = af; g1.ldd = b.s; g1.d_batch = b.s * b.s;
+                        g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.batch = C; g1.c1 = 0.f; g1.c2 = 1.f;
+                        MONA_CUDA(h, launch_sgemm(g1, stream));
+                        SgemmArgs g2{};   // B = b A + c A A
+                        g2.a = af; g2.b = af; g2.a_batch = g2.b_batch = b.s * b.s;
+                        g2.a_si = b.s; g2.a_sk = 1; g2.b_sk = b.s; g2.b_sj = 1;
+                        g2.cin = af; g2.d = bf; g2.ldd = b.s; g2.d_batch = b.s * b.s;
+                        g2.M = g2.N = g2.K = (int)b.s; g2.batch = C; g2.c1 = ns_b; g2.c2 = ns_c;
+                        MONA_CUDA(h, launch_sgemm(g2, stream));
+                        SgemmArgs g3{};   // X' = a X + B X (wide) or a X + X B (tall)
+                        if (!b.tall) {
+                            g3.a = bf; g3.a_si = b.s; g3.a_sk = 1; g3.a_batch = b.s * b.s;
+                            g3.b = xf[cur]; g3.b_sk = b.cols; g3.b_sj = 1; g3.b_batch = b.e;
+                            g3.M = (int)b.s; g3.N = (int)b.l;
+                        } else {
+                            g3.a = xf[cur]; g3.a_si = b.cols; g3.a_sk = 1; g3.a_batch = b.e;
+                            g3.b = bf; g3.b_sk = b.s; g3.b_sj = 1; g3.b_batch = b.s * b.s;
+                            g3.M = (int)b.l; g3.N = (int)b.s;
+                        }
+                        g3.K = (int)b.s; g3.cin = xf[cur]; g3.d = xf[nxt]; g3.ldd = b.cols; g3.d_batch = b.e;
+                        g3.batch = C; g3.c1 = ns_a; g3.c2 = 1.f;
+                        MONA_CUDA(h, launch_sgemm(g3, stream));
+                        h->launches += 3;
+                        h->flops_dense += (double)C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
+                    }
+                }
+                o_final = xf[T & 1];
+            }
+            if (phase_mask & 4u) {
+                MONA_CUDA(h, launch_update(ptrs, C, tc, vec4, o_final, b.e, b.slab_len, b.slabs, eta_lambda, eta_gamma, stream));
+                ++h->launches;
+            }
+        }
+    }
+    return MONA_OK;
+}
+
+mona_status mona_step(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads, void* stream) {
+    return mona_step_ex(h, hp, params, grads, nullptr, 7u, stream);
+}
+
+mona_status mona_step_host(mona_handle* h, const mona_hparams* hp, void* const* params, void* const* grads,
+                           const void* const* grads_host, void* const* params_host, void* stream_v) {
+    if (!h) return MONA_ERR_INVALID_ARG;
+    if (!params || !grads || !grads_host || !params_host) return h->fail(MONA_ERR_INVALID_ARG, "null pointer array");
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    MONA_CUDA(h, cudaSetDevice(h->device));
+    const int64_t n_desc = (int64_t)h->plan.descs.size();
+    for (int64_t i = 0; i < n_desc; ++i) {
+        const mona_matrix_desc& d = h->plan.descs[i];
+        if (!grads_host[i] || !grads[i]) return h->fail(MONA_ERR_INVALID_ARG, "grads_host[%lld] or grads[%lld] is null", (long long)i, (long long)i);
+        size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * (d.grad_dtype == MONA_BF16 ? 2 : 4);
+        MONA_CUDA(h, cudaMemcpyAsync(grads[i], grads_host[i], bytes, cudaMemcpyHostToDevice, stream));
+    }
+    mona_status st = mona_step_ex(h, hp, params, (const void* const*)grads, nullptr, 7u, stream_v);
+    if (st != MONA_OK) return st;
+    for (int64_t i = 0; i < n_desc; ++i) {
+        const mona_matrix_desc& d = h->plan.descs[i];
+        if (!params_host[i]) return h->fail(MONA_ERR_INVALID_ARG, "params_host[%lld] is null", (long long)i);
+        size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * 4;
+        MONA_CUDA(h, cudaMemcpyAsync(params_host[i], params[i], bytes, cudaMemcpyDeviceToHost, stream));
+    }
+    return MONA_OK;
+}
+
+mona_status mona_poll_status(mona_handle* h, void* stream_v, int64_t* first_bad_matrix) {
+    if (!h) return MONA_ERR_INVALID_ARG;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    MONA_CUDA(h, cudaSetDevice(h->device));
+    MONA_CUDA(h, cudaMemcpyAsync(h->host_status, h->ws + WS_STATUS_OFF, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, stream));
+    static const DeviceStatus cleared = {0u, INT_MAX, 0u, 0u};
+    MONA_CUDA(h, cudaMemcpyAsync(h->ws + WS_STATUS_OFF, &cleared, sizeof cleared, cudaMemcpyHostToDevice, stream));
+    MONA_CUDA(h, cudaStreamSynchronize(stream));
+    const DeviceStatus s = *h->host_status;
+    if (first_bad_matrix) *first_bad_matrix = (s.first_bad == INT_MAX) ? -1 : s.first_bad;
+    if (s.flags & STATUS_TIMEOUT) return h->fail(MONA_ERR_TIMEOUT, "a device-side wait ran out (site %u)", s.timeout_site);
+    if (s.flags & STATUS_NONFINITE) return h->fail(MONA_ERR_NONFINITE, "non-finite ||M||_F, first at matrix %d", s.first_bad);
+    return MONA_OK;
+}
+
+mona_status mona_state_layout(const mona_handle* h, int64_t desc, size_t* off_M, size_t* off_A, size_t* off_Gprev) {
+    if (!h || desc < 0 || desc >= (int64_t)h->plan.descs.size()) return MONA_ERR_INVALID_ARG;
+    const Bucket& b = h->plan.buckets[h->plan.desc_bucket[desc]];
+    const int64_t count = (int64_t)b.mats.size();
+    const int64_t base = b.state_off + h->plan.desc_pos[desc] * b.e;
+    if (off_M) *off_M = (size_t)base * 4;
+    if (off_A) *off_A = (size_t)(base + count * b.e) * 4;
+    if (off_Gprev) *off_Gprev = (size_t)(base + 2 * count * b.e) * 4;
+    return MONA_OK;
+}
+
+int64_t mona_last_launch_count(const mona_handle* h) { return h ? h->launches : 0; }
+
+mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* dense_equivalent) {
+    if (!h) return MONA_ERR_INVALID_ARG;
+    if (executed) *executed = h->flops_exec;
+    if (dense_equivalent) *dense_equivalent = h->flops_dense;
+    return MONA_OK;
+}
+
+const char* mona_last_error(const mona_handle* h) { return h ? h->last_error.c_str() : "null handle"; }
+
+void mona_destroy(mona_handle* h) {
+    if (!h) return;
+    if (h->side) cudaStreamDestroy(h->side);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->host_status) cudaFreeHost(h->host_status);
+    delete h;
+}
+
+}  // extern "C"

@@ -1,0 +1,145 @@
+"""CUDA library against the fp64 oracle, element by element on the same seeded inputs (through the C ABI)."""
+import pytest
+import torch
+
+import paper_2605_26842_b200 as pkg
+from tests.parity_util import TOL_O_BF16, TOL_O_FP32, TOL_STATE, TOL_W, run_case
+
+pytestmark = pytest.mark.gpu
+
+
+def check(errs, tol_o):
+    assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE and errs["Gprev"] <= TOL_STATE, errs
+    assert errs["O"] <= tol_o, errs
+    assert errs["dW"] <= max(TOL_W, tol_o), errs
+
+
+def test_config0_fp32_validation():
+    """256x512, 5 steps, fp32 validation Newton-Schulz: O within 1e-4, state within 1e-6."""
+    hp = pkg.default_hparams(ns_precision=1)
+    errs = run_case([(1, 256, 512)], steps=5, hp=hp, seed=1234)
+    check(errs, TOL_O_FP32)
+
+
+def test_config0_bf16_tensor_cores():
+    """256x512, 5 steps, bf16 operands / fp32 accumulate on tcgen05: O within 2e-2."""
+    errs = run_case([(1, 256, 512)], steps=5, seed=1234)
+    check(errs, TOL_O_BF16)
+
+
+@pytest.mark.parametrize("shape", [(1, 128, 256), (1, 256, 128), (3, 192, 320), (2, 320, 192), (1, 64, 128),
+                                   (2, 512, 1024), (2, 1024, 512), (1, 768, 2048), (1, 2048, 768), (1, 1024, 1024),
+                                   (1, 72, 200), (1, 1000, 136), (1, 2816, 1024), (1, 1024, 2816)])
+def test_tensor_core_shapes(shape):
+    """Wide, tall, square, ragged (not multiples of the 128x256 tile) and stacked shapes on the tcgen05 path."""
+    errs = run_case([shape], steps=2, seed=hash(shape) % 1000)
+    check(errs, TOL_O_BF16)
+
+
+@pytest.mark.parametrize("shape", [(1, 128, 256), (2, 320, 192), (1, 40, 72), (1, 33, 17), (1, 32, 1024), (1, 5, 3),
+                                   (1, 512, 1024)])
+def test_fp32_shapes(shape):
+    """fp32 validation mode incl. shapes that never go to the tensor cores (odd sizes, min(m,n) < 64)."""
+    hp = pkg.default_hparams(ns_precision=1)
+    errs = run_case([shape], steps=3, hp=hp, seed=7)
+    check(errs, TOL_O_FP32)
+
+
+def test_small_side_routes_to_cuda_cores_in_default_mode():
+    """Router-like 32x1024 and odd 33x17 in the default precision mode still run on the GPU (fp32 FMA path)."""
+    errs = run_case([(1, 32, 1024), (1, 33, 17)], steps=2, seed=5)
+    check(errs, TOL_O_FP32)
+
+
+def test_mixed_set_ten_steps():
+    """A small MoE-like set (stacked experts, attention, router), 10 steps: parameters within 3e-2."""
+    shapes = [(4, 256, 512), (4, 512, 256), (1, 512, 512), (1, 32, 512)]
+    errs = run_case(shapes, steps=10, seed=42)
+    check(errs, TOL_O_BF16)
+
+
+def test_bf16_gradients_and_padding():
+    errs = run_case([(3, 128, 384)], steps=3, grad_dtype=torch.bfloat16, pad=64, seed=9)
+    check(errs, TOL_O_BF16)
+
+
+def test_heavy_tailed_gradients():
+    hp = pkg.default_hparams(accel_beta=0.98, accel_alpha=-25.0)
+    errs = run_case([(2, 384, 512)], steps=4, hp=hp, rho=0.8, heavy_tail=True, seed=11)
+    check(errs, TOL_O_BF16)
+
+
+@pytest.mark.parametrize("T", [0, 1, 2, 4])
+def test_ns_step_counts(T):
+    hp = pkg.default_hparams(ns_steps=T)
+    errs = run_case([(1, 128, 256)], steps=2, hp=hp, seed=3)
+    check(errs, TOL_O_BF16)
+
+
+def test_fixed_scale_and_other_hyperparameters():
+    hp = pkg.default_hparams(scale_mode=1, scale_value=0.37, lr=5e-3, momentum=0.8, weight_decay=0.0,
+                             accel_beta=0.9, accel_alpha=-5.0)
+    errs = run_case([(1, 256, 256)], steps=3, hp=hp, seed=13)
+    check(errs, TOL_O_BF16)
+
+
+def test_nonfinite_gradient_is_reported():
+    dev = torch.device("cuda", 0)
+    p = [torch.zeros(2, 128, 128, device=dev), torch.zeros(1, 64, 64, device=dev)]
+    g = [torch.full((2, 128, 128), 1e-3, device=dev), torch.full((1, 64, 64), 1e-3, device=dev)]
+    g[0][1, 5, 7] = float("nan")
+    opt = pkg.MonaOptimizer(p)
+    opt.step(pkg.default_hparams(), p, g)
+    st, bad = opt.poll_status()
+    assert pkg.STATUS_NAMES[st] == "MONA_ERR_NONFINITE" and bad == 1
+    st, bad = opt.poll_status()          # the word is cleared by the first poll
+    assert st == 0 and bad == -1
+    opt.close()
+
+
+def test_argument_errors_on_device():
+    dev = torch.device("cuda", 0)
+    p = [torch.zeros(1, 64, 64, device=dev)]
+    g = [torch.zeros(1, 64, 64, device=dev)]
+    opt = pkg.MonaOptimizer(p)
+    hp = pkg.default_hparams()
+    with pytest.raises(pkg.MonaError) as e:
+        opt.step(hp, p, [None])
+    assert e.value.status == 1
+    mis = torch.zeros(64 * 64 + 1, device=dev)[1:].view(1, 64, 64)
+    with pytest.raises(pkg.MonaError) as e:
+        opt.step(hp, p, [mis])
+    assert e.value.status == 3
+    with pytest.raises(pkg.MonaError) as e:
+        opt.step(pkg.default_hparams(ns_precision=5), p, g)
+    assert e.value.status == 1
+    opt.close()
+
+
+def test_deterministic_and_resumable():
+    """Same inputs give bit-identical state and parameters; 4 steps equal 2 + checkpoint/restore + 2."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(5)
+    shapes = [(3, 256, 384), (1, 384, 256)]
+    W0 = [torch.randn(s, generator=gen) * 0.02 for s in shapes]
+    G = [[torch.randn(s, generator=gen) * 1e-3 for s in shapes] for _ in range(4)]
+    hp = pkg.default_hparams()
+
+    def run(split):
+        p = [w.clone().to(dev) for w in W0]
+        opt = pkg.MonaOptimizer(p)
+        for k in range(4):
+            if split and k == 2:
+                saved = opt.state.clone()
+                opt.close()
+                opt = pkg.MonaOptimizer(p)
+                opt.state.copy_(saved)
+            opt.step(hp, p, [g.to(dev) for g in G[k]])
+        torch.cuda.synchronize()
+        out = [t.clone() for t in p] + [opt.state.clone()]
+        opt.close()
+        return out
+
+    a, b, c = run(False), run(False), run(True)
+    for x, y, z in zip(a, b, c):
+        assert torch.equal(x, y) and torch.equal(x, z)
