@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the MONA optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--layers L] [--impl reference]
+
+A step is one pass of the whole hot path (fused prologue, Newton-Schulz, parameter update) over every
+matrix of a synthetic parameter set (see paper_2605_26842_b200/synth.py).  Prints ONE JSON line.
+
+Timing: CUDA events on the launching stream around each mona_step; between timed steps the gradient
+buffers advance one step of the AR(1) process and a buffer larger than L2 is rewritten (both untimed).
+The per-phase figures (prologue GB/s, Newton-Schulz TFLOP/s, update GB/s) come from extra passes that
+run one phase alone through mona_step_ex's phase mask.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mona_optimizer_steps_per_s"
+UNIT = "steps/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ts, row in self.rows:
+            if t0 is not None and not (t0 <= ts <= t1 + 0.15):
+                continue
+            f = [x.strip() for x in row.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(wl, per_shape: int = 1):
+    """Times the fp64 oracle, as it stands, on `per_shape` matrices of every distinct shape of the
+    workload (one full step each) and extrapolates to the whole set.  Returns (steps/s, description, threads)."""
+    import numpy as np
+    import oracle.mona_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = len(os.sched_getaffinity(0))
+    counts = {}
+    for s in wl.specs:
+        counts[(s.rows, s.cols)] = counts.get((s.rows, s.cols), 0) + s.batch
+    rng = np.random.default_rng(wl.seed)
+    hp = orc.Hyper(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha)
+    total, parts, spent = 0.0, [], 0.0
+    for (m, n), cnt in counts.items():
+        ts = []
+        for _ in range(per_shape):
+            W = rng.standard_normal((m, n)) * 0.02
+            G = rng.standard_normal((m, n)) * wl.sigma
+            st = orc.OracleState(m, n)
+            t0 = time.perf_counter()
+            orc.mona_step(W, G, st, hp)
+            ts.append(time.perf_counter() - t0)
+        t = sum(ts) / len(ts)
+        spent += sum(ts)
+        total += cnt * t
+        parts.append(f"{m}x{n}: {t * 1e3:.1f} ms x {cnt}")
+    desc = (f"fp64 numpy oracle, {per_shape} matrix per distinct shape, one full step each ({spent:.1f} s of CPU work), "
+            f"extrapolated by matrix count: " + "; ".join(parts))
+    return 1.0 / total, desc, threads
+
+
+def pick_workload(index, layers, free_bytes):
+    """The requested configuration, with the layer count reduced until it fits the device."""
+    from paper_2605_26842_b200 import synth
+    wl = synth.workload(index, layers)
+    note = ""
+    if layers is None and index in (1, 2, 3, 4):
+        nominal = {1: 12, 2: 16, 3: 24, 4: 8}[index]
+        L = nominal
+        # W, state, G resident + ~3 GB for workspace, generator temporaries and the L2 flush buffer
+        while L > 1 and synth.resident_bytes(synth.workload(index, L)) + (3 << 30) > free_bytes:
+            L -= 1
+        if L != nominal:
+            note = f"layer count reduced from {nominal} to {L} to fit device memory; per-matrix shapes unchanged"
+            wl = synth.workload(index, L)
+    return wl, note
+
+
+def run_reference(args):
+    """`--impl reference`: the oracle on the host cores, same metric and configuration."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2605_26842_b200 import synth
+    wl = synth.workload(args.config, args.layers)
+    vals = []
+    desc = ""
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        v, desc, threads = oracle_sample(wl, 1)
+        if i >= args.warmup:
+            vals.append(v)
+    value = len(vals) / sum(1.0 / v for v in vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "matrices": wl.n_matrices, "params": wl.n_params},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, help="parameter set 0..4 (default 3: the ~7B MoE set)")
+    ap.add_argument("--layers", type=int, default=None)
+    ap.add_argument("--impl", default="mona", choices=["mona", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--chunk-mb", type=int, default=None, help="override the L2 chunk budget (MiB)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_2605_26842_b200 as pkg
+    from paper_2605_26842_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if args.chunk_mb:
+        pkg.set_chunk_budget(args.chunk_mb << 20)
+
+    free_bytes, _ = torch.cuda.mem_get_info(dev)
+    wl, fit_note = pick_workload(args.config, args.layers, free_bytes)
+    # every rank owns an independent parameter set of this shape (weak scaling, no data-path collective)
+    params = synth.init_params(wl, dev, seed_offset=rank)
+    gp = synth.GradientProcess(wl, dev, keep_fp32_shadow=False)
+    opt = pkg.MonaOptimizer(params, grad_dtype=wl.grad_dtype, device=local_rank)
+    hp = pkg.default_hparams(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    g_elem = 2 if wl.grad_dtype == torch.bfloat16 else 4
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed_steps(n, mask=7, refresh=True):
+        evs = []
+        for _ in range(n):
+            if refresh:
+                gp.next()
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            if mask == 7:
+                opt.step(hp, params, gp.grads)
+            else:
+                opt.step_ex(hp, params, gp.grads, None, mask)
+            e1.record(stream)
+            evs.append((e0, e1))
+        torch.cuda.synchronize(dev)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    gp.next()
+    timed_steps(args.warmup)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_wall0 = time.time()
+    ms = timed_steps(args.steps)
+    t_wall1 = time.time()
+    barrier()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    st, bad = opt.poll_status()
+    if st != 0:
+        raise RuntimeError(f"device status {pkg.STATUS_NAMES[st]} at matrix {bad}")
+    launches_per_step = opt.last_launch_count()
+    flops_exec, flops_dense = opt.last_ns_flops()
+    total_ms = sum(ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * 1e3 / ms_per_step
+
+    # ---- per-phase passes (one phase alone; state keeps evolving, which does not change the work) ----
+    n_phase = max(2, min(args.steps, 3))
+    timed_steps(1, mask=1, refresh=False)
+    ms_pro = statistics.median(timed_steps(n_phase, mask=1, refresh=False))
+    timed_steps(1, mask=2, refresh=False)
+    ms_ns = statistics.median(timed_steps(n_phase, mask=2, refresh=False))
+    ns_launches = opt.last_launch_count()
+    timed_steps(1, mask=4, refresh=False)
+    ms_upd = statistics.median(timed_steps(n_phase, mask=4, refresh=False))
+    st, bad = opt.poll_status()   # phase-only passes may see stale iterates; clear whatever they latched
+
+    peaks, peak_src = load_peaks()
+    n = wl.n_params
+    pro_bytes = n * (12 + g_elem + 12 + 2)          # read G, G_prev, A, M; write G_prev, A, M, bf16 X
+    upd_bytes = n * (4 + 2 + 4)                     # read W, bf16 O; write W
+    pro_gbs = pro_bytes / (ms_pro * 1e-3) / 1e9
+    upd_gbs = upd_bytes / (ms_upd * 1e-3) / 1e9
+    ns_tflops = flops_exec / (ms_ns * 1e-3) / 1e12
+    # the Newton-Schulz GEMM kernel runs inside a long step: compare with the sustained GEMM peak
+    roofline = {"kernel": "tc_gemm_kernel (Newton-Schulz GEMMs, all launches of one step)", "bound": "tensor",
+                "achieved": ns_tflops, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": ns_tflops / peaks["bf16_tflops_sustained"], "peak_source": peak_src + " (sustained bf16 GEMM)",
+                "frac_of_burst_peak": ns_tflops / peaks["bf16_tflops"], "frac_of_nominal_2250": ns_tflops / 2250.0,
+                "flops_per_launch": flops_exec / max(1, ns_launches), "launches_per_step": ns_launches,
+                "avg_launch_us": ms_ns * 1e3 / max(1, ns_launches), "traffic": None,
+                "dense_equivalent_tflops": flops_dense / (ms_ns * 1e-3) / 1e12}
+    phases = {"prologue_ms": ms_pro, "prologue_gbs": pro_gbs, "prologue_frac_of_hbm_peak": pro_gbs / peaks["hbm_gbs"],
+              "prologue_frac_of_nominal_8000": pro_gbs / 8000.0, "prologue_bytes_per_elem": 12 + g_elem + 14,
+              "ns_ms": ms_ns, "ns_tflops_executed": ns_tflops, "update_ms": ms_upd, "update_gbs": upd_gbs,
+              "update_frac_of_hbm_peak": upd_gbs / peaks["hbm_gbs"], "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peak_src}
+
+    # ---- end to end: host gradients in, host parameters out, through mona_step_host ----
+    e2e = None
+    if not args.no_e2e:
+        try:
+            g_host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in gp.grads]
+            p_host = [torch.empty(p.shape, dtype=p.dtype, pin_memory=True) for p in params]
+            for h_, g in zip(g_host, gp.grads):
+                h_.copy_(g)
+            torch.cuda.synchronize(dev)
+            h2d = sum(g.numel() * g.element_size() for g in gp.grads)
+            d2h = sum(p.numel() * p.element_size() for p in params)
+            n_e2e = max(1, min(args.steps, 3))
+            e_ms = []
+            for i in range(1 + n_e2e):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                barrier()
+                e0.record(stream)
+                opt.step_host(hp, params, gp.grads, g_host, p_host)
+                e1.record(stream)
+                torch.cuda.synchronize(dev)
+                if i > 0:
+                    e_ms.append(e0.elapsed_time(e1))
+            e_total = sum(e_ms)
+            if dist is not None:
+                t = torch.tensor([e_total], dtype=torch.float64, device=dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                e_total = float(t.item())
+            e2e = {"value": world * 1e3 / (e_total / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                   "steps": n_e2e, "api": "mona_step_host (pinned host gradients in, updated parameters out)"}
+            del g_host, p_host
+        except Exception as exc:   # e.g. not enough pinned host memory
+            e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "error": str(exc)[:200]}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        v, desc, threads = oracle_sample(wl, 1)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16 tensor-core Newton-Schulz with fp32 accumulate; fp32 state and parameters",
+                "data": "synthetic",
+                "config": {"workload": wl.name, "config_index": args.config, "matrices": wl.n_matrices, "params": wl.n_params,
+                           "grad_dtype": str(wl.grad_dtype).replace("torch.", ""), "gradient_process":
+                           f"AR(1) rho={wl.rho} sigma={wl.sigma} {wl.dist}", "ns_steps": hp.ns_steps,
+                           "accel_beta": wl.accel_beta, "accel_alpha": wl.accel_alpha, "parallelism":
+                           "independent parameter set per GPU, no collective" if world > 1 else "single GPU",
+                           "l2": "inputs larger than L2 and a 256 MiB buffer rewritten between timed steps",
+                           "timing": "CUDA events around each mona_step; gradient refresh between steps untimed",
+                           "note": fit_note},
+                "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
+                "step_ms_each": ms, "clocks": clocks, "roofline": roofline, "phases": phases, "e2e": e2e, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    opt.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
