@@ -153,6 +153,32 @@ int64_t mona_last_launch_count(const mona_handle* h);
  * (4 s^2 l + 2 s^3 per matrix and iteration).  Either pointer may be NULL. */
 mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* dense_equivalent);
 
+/* Allocation-free prologue for ONE matrix.  The paper has no counterpart to this entry point; it exists
+ * for integration reasons only.  It performs lines 4-7 and 10 of Algorithm 1 on a rows x cols matrix
+ * (A, M, G_prev updated in place from `grad`, all device pointers, 16-byte aligned, dense row-major),
+ * writes 1 / (||M_k||_F + eps) to inv_norm_out[0] (device) and, when xhat_bf16 is not NULL, the bf16
+ * copy of M_k there.  Results equal those of the prologue phase of mona_step_ex().
+ *
+ * Who needs it: callers that cannot get device memory when they call us - for instance a trainer whose
+ * framework allocator already owns all of HBM, or a hook running where the device-wide stall of
+ * cudaMalloc/cudaFree is not acceptable.  This function calls no allocator of any kind.  The few hundred
+ * scratch words the reduction needs (slab partial sums and an arrival counter) sit in a 2 KiB array
+ * compiled into the library, resident on every GPU that loads the library until the process ends.
+ *
+ * Limits and rules:
+ *   - rows * cols <= 16,777,216 (one 4096 x 4096 matrix); larger inputs are refused with
+ *     MONA_ERR_UNSUPPORTED_SHAPE and an explanatory message in `err`.
+ *   - It works on the CURRENT device; all pointers must belong to it.  The first call on each device
+ *     looks up the device address of the built-in array; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents (the function
+ *     re-zeroes the counter it depends on).  Two calls whose kernels may overlap on the GPU - different
+ *     streams, no ordering between them - race on it; order them yourself.
+ *   - `err` (may be NULL) receives a NUL-terminated message of at most err_len bytes.
+ * Enqueued on `stream`; does not synchronise. */
+mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtype, float* M, float* A, float* G_prev,
+                                  void* xhat_bf16, float* inv_norm_out, int64_t rows, int64_t cols,
+                                  const mona_hparams* hp, void* stream, char* err, size_t err_len);
+
 /* Human-readable detail of the last failing call on this handle (never NULL). */
 const char* mona_last_error(const mona_handle* h);
 

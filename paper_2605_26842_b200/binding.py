@@ -198,3 +198,22 @@ class MonaOptimizer:
             self.close()
         except Exception:
             pass
+
+
+def prologue_noalloc(grad: torch.Tensor, M: torch.Tensor, A: torch.Tensor, G_prev: torch.Tensor,
+                     inv_norm_out: torch.Tensor, hp: Hparams, xhat: Optional[torch.Tensor] = None):
+    """mona_prologue_noalloc on the current device and current torch stream: the fused prologue for one
+    (rows, cols) matrix for callers that cannot allocate device memory.  Raises MonaError with the
+    library's message on refusal (e.g. a matrix beyond the built-in scratch limit)."""
+    L = lib()
+    fn = L.mona_prologue_noalloc
+    fn.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                   C.POINTER(Hparams), C.c_void_p, C.c_char_p, C.c_size_t]
+    fn.restype = C.c_int
+    rows, cols = grad.shape[-2], grad.shape[-1]
+    err = C.create_string_buffer(256)
+    st = fn(grad.data_ptr(), MONA_BF16 if grad.dtype == torch.bfloat16 else MONA_F32, M.data_ptr(), A.data_ptr(),
+            G_prev.data_ptr(), None if xhat is None else xhat.data_ptr(), inv_norm_out.data_ptr(), rows, cols, C.byref(hp),
+            C.c_void_p(torch.cuda.current_stream().cuda_stream), err, len(err))
+    if st:
+        raise MonaError(st, err.value.decode())

@@ -238,3 +238,108 @@ cudaError_t launch_scale(const float* M, float* X, const float* inv_norm, int C,
 }
 
 }  // namespace mona
+
+// ---------------------------------------------------------------------------------------------------
+// Allocation-free single-matrix prologue (mona_prologue_noalloc, declared in include/mona.h).
+//
+// The fused prologue needs a little global scratch: one partial sum of squares per slab and a counter
+// that tells the last slab to finish that it must add them up.  The handle-based path keeps that
+// scratch in the caller's workspace.  Some callers have no workspace to give and cannot create one:
+// a process whose framework allocator has already claimed the whole device, or a hook that must not
+// trigger the device-wide synchronisation that cudaMalloc/cudaFree imply.  For them the scratch below
+// lives in the library image itself; every GPU that loads the library carries these 2 KiB until the
+// process exits.
+#include <mutex>
+
+#include "../../include/mona.h"
+
+namespace mona {
+namespace {
+
+constexpr long long NOALLOC_MAX_ELEMS = 1ll << 24;      // one 4096 x 4096 matrix
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+struct NoAllocScratch {
+    float partials[MAX_SLABS];     // slab sums of squares (fully rewritten by every call)
+    unsigned int counter;          // slab arrival counter; must be 0 when a call starts
+    unsigned int pad[3];
+    DeviceStatus status;           // non-finite flag sink (not reported by this entry point)
+};
+static_assert(sizeof(NoAllocScratch) <= 2048, "scratch layout");
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never an address to hand to a kernel.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[2048];
+
+std::mutex g_noalloc_mutex;
+NoAllocScratch* g_noalloc_dev_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
+
+void set_msg(char* buf, size_t len, const char* msg) {
+    if (buf && len) {
+        size_t i = 0;
+        for (; msg[i] && i + 1 < len; ++i) buf[i] = msg[i];
+        buf[i] = 0;
+    }
+}
+
+F2 split_double(double v) {
+    F2 r;
+    r.hi = (float)v;
+    r.lo = (float)(v - (double)r.hi);
+    return r;
+}
+
+}  // namespace
+}  // namespace mona
+
+extern "C" mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtype, float* M, float* A, float* G_prev,
+                                             void* xhat_bf16, float* inv_norm_out, int64_t rows, int64_t cols,
+                                             const mona_hparams* hp, void* stream_v, char* err, size_t err_len) {
+    using namespace mona;
+    if (!grad || !M || !A || !G_prev || !inv_norm_out || !hp) { set_msg(err, err_len, "null pointer argument"); return MONA_ERR_INVALID_ARG; }
+    if (rows <= 0 || cols <= 0) { set_msg(err, err_len, "rows and cols must be positive"); return MONA_ERR_INVALID_ARG; }
+    if (grad_dtype != MONA_F32 && grad_dtype != MONA_BF16) { set_msg(err, err_len, "unknown grad_dtype"); return MONA_ERR_INVALID_ARG; }
+    if (rows > NOALLOC_MAX_ELEMS || cols > NOALLOC_MAX_ELEMS || rows * cols > NOALLOC_MAX_ELEMS) {
+        set_msg(err, err_len, "matrix larger than the built-in scratch supports: rows*cols must be <= 16777216 (4096 x 4096)");
+        return MONA_ERR_UNSUPPORTED_SHAPE;
+    }
+    if (((uintptr_t)grad | (uintptr_t)M | (uintptr_t)A | (uintptr_t)G_prev | (uintptr_t)xhat_bf16) & 15) {
+        set_msg(err, err_len, "matrix pointers must be 16-byte aligned");
+        return MONA_ERR_ALIGNMENT;
+    }
+    int dev = -1;
+    cudaError_t ce = cudaGetDevice(&dev);
+    if (ce != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) { set_msg(err, err_len, "no current CUDA device"); return MONA_ERR_CUDA; }
+    NoAllocScratch* scratch = nullptr;
+    {
+        // once per device, with that device current: resolve the device address of the static array
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_dev_ptr[dev]) {
+            void* p = nullptr;
+            ce = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            if (ce != cudaSuccess || !p) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
+            g_noalloc_dev_ptr[dev] = reinterpret_cast<NoAllocScratch*>(p);
+        }
+        scratch = g_noalloc_dev_ptr[dev];
+    }
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    const long long e = rows * cols;
+    long long slab = 16384;
+    if ((e + slab - 1) / slab > MAX_SLABS) slab = ((e + MAX_SLABS - 1) / MAX_SLABS + 1023) / 1024 * 1024;
+    const int slabs = (int)((e + slab - 1) / slab);
+    // the array keeps whatever the previous call left: the counter has to start from zero
+    ce = cudaMemsetAsync(&scratch->counter, 0, sizeof(unsigned int), stream);
+    if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
+    ChunkPtrs ptrs;
+    ptrs.g[0] = grad; ptrs.w[0] = nullptr; ptrs.o[0] = nullptr; ptrs.gid[0] = 0;
+    PrologueScalars k;
+    k.beta = split_double(hp->accel_beta);
+    k.one_minus_beta = split_double(1.0 - hp->accel_beta);
+    k.alpha = split_double(hp->accel_alpha);
+    k.mu = split_double(hp->momentum);
+    k.eps = (float)hp->norm_eps;
+    ce = launch_prologue(ptrs, 1, grad_dtype == MONA_BF16, e % 4 == 0, M, A, G_prev, (__nv_bfloat16*)xhat_bf16, scratch->partials,
+                         &scratch->counter, inv_norm_out, &scratch->status, e, slab, slabs, k, stream);
+    if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
+    set_msg(err, err_len, "");
+    return MONA_OK;
+}
