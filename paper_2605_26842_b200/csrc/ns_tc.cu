@@ -3,8 +3,8 @@
 // One persistent CTA per SM walks a static list of output tiles (128 x up-to-256) of all matrices of
 // a chunk.  Warp 0 stages bf16 operand tiles with TMA into a 4-deep shared-memory ring, warp 1 issues
 // tcgen05.mma (fp32 accumulators in tensor memory, two accumulator buffers so the epilogue of one tile
-// overlaps the main loop of the next), warps 2-5 read the accumulator back with tcgen05.ld, apply the
-// polynomial term (b A + c A^2, a X + B X) and the deferred 1/||M||_F scale, and store bf16.
+// overlaps the main loop of the next), warps 2-9 read the accumulator back with tcgen05.ld, apply the
+// polynomial term (b A + c A^2 + a I) and the deferred 1/||M||_F scale, and store bf16.
 //
 // Every wait is bounded: a wait that runs out latches STATUS_TIMEOUT, raises a CTA-wide abort flag, and
 // all roles fall through to the common exit where tensor memory is released.
@@ -14,7 +14,8 @@ namespace mona {
 
 namespace {
 
-constexpr int TC_THREADS = 192;
+constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
+constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
 constexpr uint32_t A_STAGE_BYTES = TC_BM * TC_BK * 2;            // 16 KiB
 constexpr uint32_t B_STAGE_BYTES = TC_BN * TC_BK * 2;            // 32 KiB
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KiB
@@ -199,7 +200,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, TC_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_b) : "memory");
@@ -275,60 +276,85 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
             }
         }
     } else {
-        // ---------------- epilogue (warps 2..5) ----------------
-        const int quad = warp & 3;                       // tensor-memory lane quadrant this warp may read
+        // ---------------- epilogue (warps 2..9) ----------------
+        // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4); the two warps
+        // of a quadrant take alternate 32-column chunks.  Two chunks are in flight per warp so that the
+        // tensor-memory load of one overlaps the arithmetic and stores of the other.
+        const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row_in_tile = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         uint32_t acc = 0, acc_phase = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
             const TileCoord tc = decode_tile(g, t);
-            bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, status, 4);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
             const int gr = tc.tm * TC_BM + row_in_tile;
             const int n0 = tc.tn * TC_BN;
             const bool row_ok = gr < g.M;
             const long long mat_off = (long long)tc.c * g.mat_stride;
+            const long long row_off = mat_off + (long long)gr * g.ld;
             float post = 1.0f;
-            if (g.post_mode) { float s = g.inv_norm[tc.c]; post = g.post_mode == 2 ? s * s : s; }
-            const float c1 = g.c1, c2 = g.c2;
-            for (int col0 = 0; col0 < tc.nw; col0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + acc * TC_BN + col0, v);
+            if (g.post_mode) { float sc = g.inv_norm[tc.c]; post = g.post_mode == 2 ? sc * sc : sc; }
+            const float c1 = g.c1, c2 = g.c2 * post;
+            const int nchunks = tc.nw >> 5;
+            // operand of the axpy term for the first pair of chunks, requested before the accumulator is ready
+            uint4 cin_raw[2][4];
+            auto load_cin = [&](int ch, uint4* dst) {
+                const int gc0 = n0 + ch * 32;
+                #pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (row_ok && ch < nchunks && gc0 + 8 * q < g.N) dst[q] = *reinterpret_cast<const uint4*>(g.cin + row_off + gc0 + 8 * q);
+                    else dst[q] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            };
+            if (g.cin) { load_cin(half, cin_raw[0]); load_cin(half + 2, cin_raw[1]); }
+            bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, status, 4);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_base = tmem_base + lane_base + acc * TC_BN;
+            for (int ch0 = half; ch0 < nchunks; ch0 += 4) {
+                const int ch1 = ch0 + 2;
+                float v[2][32];
+                tmem_ld32(t_base + ch0 * 32, v[0]);
+                if (ch1 < nchunks) tmem_ld32(t_base + ch1 * 32, v[1]);
                 tmem_ld_wait();
-                const int gc0 = n0 + col0;
-                if (row_ok && gc0 < g.N) {
-                    const long long off = mat_off + (long long)gr * g.ld + gc0;
-                    if (g.cin) {
-                        #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            if (gc0 + 8 * q < g.N) {
-                                uint4 raw = *reinterpret_cast<const uint4*>(g.cin + off + 8 * q);
-                                const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-                                #pragma unroll
-                                for (int h = 0; h < 4; ++h) {
-                                    float lo = __uint_as_float(w[h] << 16), hi = __uint_as_float(w[h] & 0xffff0000u);
-                                    v[8 * q + 2 * h] = post * fmaf(c1, lo, c2 * v[8 * q + 2 * h]);
-                                    v[8 * q + 2 * h + 1] = post * fmaf(c1, hi, c2 * v[8 * q + 2 * h + 1]);
-                                }
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int ch = u == 0 ? ch0 : ch1;
+                    const int gc0 = n0 + ch * 32;
+                    if (ch < nchunks && row_ok && gc0 < g.N) {
+                        float* vv = v[u];
+                        if (g.cin) {
+                            const uint32_t w[16] = {cin_raw[u][0].x, cin_raw[u][0].y, cin_raw[u][0].z, cin_raw[u][0].w,
+                                                    cin_raw[u][1].x, cin_raw[u][1].y, cin_raw[u][1].z, cin_raw[u][1].w,
+                                                    cin_raw[u][2].x, cin_raw[u][2].y, cin_raw[u][2].z, cin_raw[u][2].w,
+                                                    cin_raw[u][3].x, cin_raw[u][3].y, cin_raw[u][3].z, cin_raw[u][3].w};
+                            #pragma unroll
+                            for (int h = 0; h < 16; ++h) {
+                                vv[2 * h] = fmaf(c1 * post, __uint_as_float(w[h] << 16), c2 * vv[2 * h]);
+                                vv[2 * h + 1] = fmaf(c1 * post, __uint_as_float(w[h] & 0xffff0000u), c2 * vv[2 * h + 1]);
                             }
+                        } else {
+                            #pragma unroll
+                            for (int j = 0; j < 32; ++j) vv[j] *= c2;
                         }
-                    } else {
-                        const float s = post * c2;
+                        if (g.diag_add != 0.f && gr >= gc0 && gr < gc0 + 32) {
+                            #pragma unroll
+                            for (int j = 0; j < 32; ++j) vv[j] += (gc0 + j == gr) ? g.diag_add : 0.f;
+                        }
                         #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] *= s;
-                    }
-                    #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        if (gc0 + 8 * q < g.N) *reinterpret_cast<uint4*>(g.out + off + 8 * q) = pack8(v + 8 * q);
-                    if (g.symmetric && (gc0 / TC_BM) < tc.tm) {
-                        // strictly-lower 128-block: the transposed block is not computed anywhere, write it here
-                        __nv_bfloat16* col = g.out + mat_off + (long long)gc0 * g.ld + gr;
-                        #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (gc0 + j < g.N) col[(long long)j * g.ld] = __float2bfloat16_rn(v[j]);
+                        for (int q = 0; q < 4; ++q)
+                            if (gc0 + 8 * q < g.N) *reinterpret_cast<uint4*>(g.out + row_off + gc0 + 8 * q) = pack8(vv + 8 * q);
+                        if (g.symmetric && (gc0 / TC_BM) < tc.tm) {
+                            // strictly-lower 128-block: the transposed block is not computed anywhere, write it here
+                            __nv_bfloat16* col = g.out + mat_off + (long long)gc0 * g.ld + gr;
+                            #pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (gc0 + j < g.N) col[(long long)j * g.ld] = __float2bfloat16_rn(vv[j]);
+                        }
                     }
                 }
+                if (g.cin && ch0 + 4 < nchunks) { load_cin(ch0 + 4, cin_raw[0]); load_cin(ch0 + 6, cin_raw[1]); }
             }
             tc_fence_before();
             __syncwarp();

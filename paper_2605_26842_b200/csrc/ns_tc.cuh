@@ -14,7 +14,7 @@ constexpr int TC_BOX = 64;      // every TMA box is 64 (contiguous) x 64 (stride
 constexpr int TC_STAGES = 4;
 
 // One batched GEMM of the iteration of Eq. newton_schulz over the C matrices of a chunk:
-//     D = post * (c1 * Cin + c2 * Aop x Bop^T),   D, Cin bf16; accumulation fp32.
+//     D = post * (c1 * Cin + c2 * Aop x Bop^T) + diag_add * I,   D, Cin bf16; accumulation fp32.
 // Operand tiles come through the two tensor maps.  An operand is "K-major" when k is its contiguous
 // index (tensor map dims {K, rows, C}) and "MN-major" when its row index is contiguous (dims {rows, K, C});
 // tall weights use the MN-major form so that X^T X and B X need no transposed copy.
@@ -30,6 +30,7 @@ struct TcGemm {
     __nv_bfloat16* out;
     long long ld, mat_stride;   // leading dimension and per-matrix stride of cin/out, in elements
     float c1, c2;
+    float diag_add;             // added to D(i,i): folds the a*X term of the quintic into B' = b A + c A^2 + a I
     const float* inv_norm;      // per-matrix 1/(||M||_F + eps), used when post_mode != 0
     int post_mode;              // 0: post = 1, 1: post = inv, 2: post = inv^2
 };

@@ -45,9 +45,10 @@ def test_fp32_shapes(shape):
     check(errs, TOL_O_FP32)
 
 
-def test_small_side_routes_to_cuda_cores_in_default_mode():
-    """Router-like 32x1024 and odd 33x17 in the default precision mode still run on the GPU (fp32 FMA path)."""
-    errs = run_case([(1, 32, 1024), (1, 33, 17)], steps=2, seed=5)
+def test_small_and_odd_shapes_in_default_mode():
+    """Router-like 32x1024 (shorter side < 64), 33x17 (sides not a multiple of 8) and 8x24 take the fp32 FMA
+    path in the default precision mode too: everything still runs on the GPU, to the fp32 tolerance."""
+    errs = run_case([(1, 32, 1024), (1, 33, 17), (1, 8, 24)], steps=2, seed=5)
     check(errs, TOL_O_FP32)
 
 
