@@ -162,7 +162,7 @@ F2 split(double v) {
 
 struct mona_handle {
     Plan plan;
-    int device = 0, num_sms = 0;
+    int device = 0, num_sms = 0, max_pairs = 0;
     uint8_t* state = nullptr;
     uint8_t* ws = nullptr;
     cudaStream_t side = nullptr;
@@ -253,7 +253,7 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
         ok = ok && encode_map(encode, &b.tm_b, h->ws + b.off_b, b.s, b.s, b.Cb);
         if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
     }
-    MONA_CUDA(h, tc_gemm_configure());
+    MONA_CUDA(h, tc_gemm_configure(&h->max_pairs));
     MONA_CUDA(h, cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
     MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
     MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
@@ -331,7 +331,6 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             float* Gc = Gst + start * b.e;
             __nv_bfloat16* xb[2] = {(__nv_bfloat16*)(h->ws + b.off_x[0]), (__nv_bfloat16*)(h->ws + b.off_x[1])};
             __nv_bfloat16* ab = (__nv_bfloat16*)(h->ws + b.off_a);
-            __nv_bfloat16* bb = (__nv_bfloat16*)(h->ws + b.off_b);
             float* xf[2] = {(float*)(h->ws + b.off32_x[0]), (float*)(h->ws + b.off32_x[1])};
             float* af = (float*)(h->ws + b.off32_a);
             float* bf = (float*)(h->ws + b.off32_b);
@@ -346,30 +345,30 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                 if (phase_mask & 2u) {
                     for (int t = 0; t < T; ++t) {
                         const int cur = t & 1, nxt = cur ^ 1;
-                        TcGemm g1{};
+                        TcGemm g1{};     // A = X X^T (wide) or X^T X (tall): lower-triangle tiles only
                         g1.C = C; g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_mn = g1.b_mn = b.tall ? 1 : 0; g1.symmetric = 1;
-                        g1.cin = nullptr; g1.out = ab; g1.ld = b.s; g1.mat_stride = b.s * b.s; g1.c1 = 0.f; g1.c2 = 1.f;
+                        g1.cin = nullptr; g1.c1 = 0.f; g1.c2 = 1.f;
                         g1.inv_norm = inv_norm; g1.post_mode = t == 0 ? 2 : 0;
                         tc_gemm_plan(g1);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_x[cur], g1, h->num_sms, dstatus, stream));
-                        TcGemm g2{};
-                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_mn = g2.b_mn = 0; g2.symmetric = 1;
-                        g2.cin = ab; g2.out = bb; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
-                        g2.inv_norm = inv_norm; g2.post_mode = 0; g2.diag_add = ns_a;   // B' = b A + c A^2 + a I
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_x[cur], b.tm_a, g1, h->max_pairs, dstatus, stream));
+                        TcGemm g2{};     // B' = b A + c A A + a I, operands and result lower-block-stored
+                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1;
+                        g2.cin = ab; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
+                        g2.inv_norm = inv_norm; g2.post_mode = 0; g2.diag_add = ns_a;
                         tc_gemm_plan(g2);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_a, b.tm_a, g2, h->num_sms, dstatus, stream));
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_a, b.tm_a, b.tm_b, g2, h->max_pairs, dstatus, stream));
                         TcGemm g3{};
                         g3.C = C; g3.K = (int)b.s; g3.symmetric = 0;
-                        g3.cin = nullptr; g3.out = xb[nxt]; g3.ld = b.cols; g3.mat_stride = b.e; g3.c1 = 0.f; g3.c2 = 1.f;
+                        g3.cin = nullptr; g3.c1 = 0.f; g3.c2 = 1.f;
                         g3.inv_norm = inv_norm; g3.post_mode = t == 0 ? 1 : 0;
-                        if (!b.tall) {   // X' = (a I + B) X : B' is the K-major "A" operand, X the MN-major "B" operand
-                            g3.M = (int)b.s; g3.N = (int)b.l; g3.a_mn = 0; g3.b_mn = 1;
+                        if (!b.tall) {   // X' = B' X : B' is the symmetric "A" operand, X the MN-major "B" operand
+                            g3.M = (int)b.s; g3.N = (int)b.l; g3.a_sym = 1; g3.b_mn = 1;
                             tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_b, b.tm_x[cur], g3, h->num_sms, dstatus, stream));
-                        } else {         // X' = X (a I + B) : X is K-major, B' (symmetric) serves as its own transpose
-                            g3.M = (int)b.l; g3.N = (int)b.s; g3.a_mn = 0; g3.b_mn = 0;
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_b, b.tm_x[cur], b.tm_x[nxt], g3, h->max_pairs, dstatus, stream));
+                        } else {         // X' = X B' : X is K-major, the symmetric B' serves as its own transpose
+                            g3.M = (int)b.l; g3.N = (int)b.s; g3.a_mn = 0; g3.b_sym = 1;
                             tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_b, g3, h->num_sms, dstatus, stream));
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_b, b.tm_x[nxt], g3, h->max_pairs, dstatus, stream));
                         }
                         h->launches += 3;
                         h->flops_exec += tc_gemm_executed_flops(g1) + tc_gemm_executed_flops(g2) + tc_gemm_executed_flops(g3);

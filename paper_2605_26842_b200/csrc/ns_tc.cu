@@ -1,42 +1,80 @@
 // Tensor-core GEMMs of the Newton-Schulz iteration (Eq. newton_schulz) for sm_100a.
 //
-// One persistent CTA per SM walks a static list of output tiles (128 x up-to-256) of all matrices of
-// a chunk.  Warp 0 stages bf16 operand tiles with TMA into a 4-deep shared-memory ring, warp 1 issues
-// tcgen05.mma (fp32 accumulators in tensor memory, two accumulator buffers so the epilogue of one tile
-// overlaps the main loop of the next), warps 2-9 read the accumulator back with tcgen05.ld, apply the
-// polynomial term (b A + c A^2 + a I) and the deferred 1/||M||_F scale, and store bf16.
+// The kernel is persistent and runs as clusters of two CTAs on neighbouring SMs.  A CTA pair walks a
+// static list of 256 x 256 output tiles of all matrices of a chunk; one tcgen05.mma.cta_group::2
+// instruction stream, issued by the even CTA (the "leader"), drives the tensor cores of both SMs.
+// Each CTA stages its own 128 rows of the A operand and its own 128 rows of the B operand per k-slice,
+// so a pair moves 64 KiB from L2 per 256 x 256 x 64 step (half of what two independent 128 x 256 tiles
+// would).  Roles inside a CTA:
+//   warp 0     TMA producer: operand boxes into a ring of shared-memory stages; the copies of both CTAs
+//              complete on the leader's "full" barrier,
+//   warp 1     owner of tensor memory; in the leader its lane 0 issues the MMAs and commits them to
+//              the "empty" barriers of both CTAs (multicast commit),
+//   warps 2-9  epilogue: tcgen05.ld the CTA's 128 x 256 fp32 accumulator, apply the polynomial term
+//              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, pack to bf16 into swizzled
+//              shared memory and hand the boxes to TMA stores.
+// Two accumulators (2 x 256 tensor-memory columns) let the epilogue of one tile overlap the main loop
+// of the next.
 //
-// Every wait is bounded: a wait that runs out latches STATUS_TIMEOUT, raises a CTA-wide abort flag, and
-// all roles fall through to the common exit where tensor memory is released.
+// Every wait on an mbarrier is bounded: when one runs out the CTA latches STATUS_TIMEOUT, raises its
+// abort flag, and all roles fall through to the common exit, where tensor memory is released.
 #include "ns_tc.cuh"
 
 namespace mona {
 
 namespace {
 
+constexpr int TC_STAGES = 5;
+constexpr int TC_EPI_BUFS = 2;
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
-constexpr int TC_THREADS = 64 + 32 * TC_EPI_WARPS;
-constexpr uint32_t A_STAGE_BYTES = TC_BM * TC_BK * 2;            // 16 KiB
-constexpr uint32_t B_STAGE_BYTES = TC_BN * TC_BK * 2;            // 32 KiB
-constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;  // 48 KiB
-constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;              // 8 KiB
-constexpr uint32_t TMEM_COLS = 512;                              // 2 accumulators x 256 fp32 columns
+constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
+constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
+constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
+constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows staged by one CTA
+constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
+constexpr uint32_t A_STAGE_BYTES = CTA_M * TC_BK * 2;             // 16 KiB
+constexpr uint32_t B_STAGE_BYTES = CTA_N * TC_BK * 2;             // 16 KiB
+constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // 32 KiB per CTA
+constexpr uint32_t STAGE_TX_BYTES = 2 * STAGE_BYTES;              // both CTAs' copies land on the leader's barrier
+constexpr int EPI_COLS = 128;                                     // output columns per epilogue phase
+constexpr uint32_t EPI_BUF_BYTES = CTA_M * EPI_COLS * 2;          // 32 KiB = 2 x 2 boxes
+constexpr uint32_t TMEM_COLS = 512;                               // 2 accumulators x 256 fp32 columns
 constexpr uint32_t SMEM_CTRL_BYTES = 256;
-constexpr uint32_t SMEM_TOTAL = TC_STAGES * STAGE_BYTES + SMEM_CTRL_BYTES + 1024;  // +1024: manual alignment
-constexpr long long WAIT_BUDGET_CYCLES = 4000000000ll;           // ~2 s
+constexpr uint32_t SMEM_TOTAL = TC_STAGES * STAGE_BYTES + TC_EPI_BUFS * EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
+constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
+static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
+static_assert(8 * (2 * TC_STAGES + 4) + 8 <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// ---- cluster --------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 // ---- mbarrier -------------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.shared::cta.b64 st, [%0];\n\t}" ::"r"(bar) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes)
                  : "memory");
+}
+// Arrive on a barrier given by its cluster-wide address (own CTA or the peer).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -69,36 +107,70 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// ---- named barriers among the epilogue warps ------------------------------------------------------
+__device__ __forceinline__ void epi_bar_sync(int id) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(TC_EPI_THREADS) : "memory");
+}
+// Barrier + AND-reduction of a predicate over the epilogue threads (same answer in every thread).
+__device__ __forceinline__ bool epi_bar_all(int id, bool pred) {
+    uint32_t in = pred ? 1u : 0u, out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "barrier.cta.red.and.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out)
+        : "r"(in), "r"(id), "r"(TC_EPI_THREADS)
+        : "memory");
+    return out != 0;
+}
+
 // ---- TMA ------------------------------------------------------------------------------------------
+// Box load into this CTA's shared memory; completion bytes are counted on `bar`, a cluster-wide
+// address that may name the barrier of the peer CTA of the pair (cta_group::2 form).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- tcgen05 --------------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// Arrives (once the MMAs issued so far have completed) on the barrier at offset `bar` in both CTAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask)
+                 : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate; accumulate == 0 overwrites D.
+// D[tmem] (+)= A[smem] * B[smem]^T over the CTA pair, bf16 inputs, fp32 accumulate; accumulate == 0 overwrites D.
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
@@ -133,40 +205,38 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
     d |= (uint64_t)2 << 61;                                                  // layout: 128-byte swizzle
     return d;
 }
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn, int b_mn) {
+// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 256 over the pair, N = 256.
+__device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn) {
     return (1u << 4)                      // D format fp32
            | (1u << 7) | (1u << 10)       // A, B format bf16
            | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
-           | ((uint32_t)(n >> 3) << 17)
+           | ((uint32_t)(TC_BN >> 3) << 17)
            | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
 struct TileCoord {
-    int c, tm, tn, nw;   // matrix, tile row, tile column, columns of this tile (multiple of 64, <= 256)
+    int c, tm, tn;   // matrix, tile row, tile column
 };
 
 __device__ __forceinline__ TileCoord decode_tile(const TcGemm& g, int t) {
     TileCoord tc;
     tc.c = t / g.tiles_per_mat;
-    int r = t - tc.c * g.tiles_per_mat;
-    int n_left;
+    const int r = t - tc.c * g.tiles_per_mat;
     if (g.symmetric) {
-        // rows come in pairs (2q, 2q+1), each row of the pair owning q+1 tiles of width 256
-        int q = 0;
-        while ((q + 1) * (q + 2) <= r) ++q;
-        int rr = r - q * (q + 1);
-        if (rr >= q + 1) { tc.tm = 2 * q + 1; tc.tn = rr - (q + 1); } else { tc.tm = 2 * q; tc.tn = rr; }
-        n_left = min(g.N, TC_BM * (tc.tm + 1)) - tc.tn * TC_BN;   // nothing right of the diagonal 128-block
+        int tm = 0;
+        while ((tm + 1) * (tm + 2) / 2 <= r) ++tm;     // lower triangle, row by row
+        tc.tm = tm;
+        tc.tn = r - tm * (tm + 1) / 2;
     } else {
         tc.tm = r / g.tiles_n;
         tc.tn = r - tc.tm * g.tiles_n;
-        n_left = g.N - tc.tn * TC_BN;
     }
-    int nw = (n_left + TC_BOX - 1) / TC_BOX * TC_BOX;
-    tc.nw = nw < TC_BN ? nw : TC_BN;
     return tc;
 }
+
+// A symmetric operand is stored as its lower block triangle: the k-slice [k0, k0 + 64) of row block
+// `blk` lies above the diagonal block exactly when it starts at or beyond the end of that block.
+__device__ __forceinline__ int fetch_transposed(int sym, int blk, int k0) { return sym && k0 >= (blk + 1) * TC_BM; }
 
 __device__ __forceinline__ uint4 pack8(const float* v) {
     uint4 r;
@@ -178,32 +248,36 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
     return r;
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b, TcGemm g,
-               DeviceStatus* __restrict__ status) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
+               const __grid_constant__ CUtensorMap tma_d, TcGemm g, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzle atoms need 1024-byte alignment
-    const uint32_t ctrl = base + TC_STAGES * STAGE_BYTES;
-    const uint32_t bar_full = ctrl;                     // TC_STAGES x 8 B
-    const uint32_t bar_empty = ctrl + 8 * TC_STAGES;    // TC_STAGES x 8 B
+    const uint32_t epi_base = base + TC_STAGES * STAGE_BYTES;
+    const uint32_t ctrl = epi_base + TC_EPI_BUFS * EPI_BUF_BYTES;
+    const uint32_t bar_full = ctrl;                             // TC_STAGES x 8 B (used in the leader)
+    const uint32_t bar_empty = ctrl + 8 * TC_STAGES;            // TC_STAGES x 8 B
     const uint32_t bar_acc_full = ctrl + 16 * TC_STAGES;        // 2 x 8 B
-    const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B
+    const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B (used in the leader)
     const uint32_t tmem_slot = bar_acc_empty + 16;              // 4 B
     uint8_t* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + (tmem_slot - ctrl));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + (tmem_slot - ctrl) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                    // 0: leader, 1: peer
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int total_tiles = g.C * g.tiles_per_mat;
     const int num_kb = (g.K + TC_BK - 1) / TC_BK;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, TC_EPI_WARPS); }
+        for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_b) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_d) : "memory");
     }
     if (warp == 1) {
         __syncwarp();
@@ -212,160 +286,189 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                    // both CTAs' barriers exist before either side signals the other
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (both CTAs) ----------------
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const uint32_t full_leader = map_to_cta(bar_full, 0);
+            for (int t = pair; t < total_tiles && ok; t += num_pairs) {
                 const TileCoord tc = decode_tile(g, t);
-                const int m0 = tc.tm * TC_BM, n0 = tc.tn * TC_BN;
-                const int nbox_b = tc.nw / TC_BOX;
-                const uint32_t tx_bytes = A_STAGE_BYTES + (uint32_t)nbox_b * BOX_BYTES;
+                const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;      // this CTA's rows of the A operand
+                const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1))) break;
-                    const uint32_t full = bar_full + 8 * stage;
+                    const uint32_t full = full_leader + 8 * stage;
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const int k0 = kb * TC_BK;
-                    mbar_arrive_expect_tx(full, tx_bytes);
+                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, STAGE_TX_BYTES);
+                    const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
+                    const int b_mn = g.b_sym ? fetch_transposed(1, tc.tn, k0) : g.b_mn;
                     #pragma unroll
-                    for (int j = 0; j < TC_BM / TC_BOX; ++j) {
-                        if (g.a_mn) tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, m0 + j * TC_BOX, k0, tc.c);
-                        else        tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, k0, m0 + j * TC_BOX, tc.c);
+                    for (int j = 0; j < CTA_M / TC_BOX; ++j) {
+                        if (a_mn) tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, m0 + j * TC_BOX, k0, tc.c);
+                        else      tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, k0, m0 + j * TC_BOX, tc.c);
                     }
-                    for (int j = 0; j < nbox_b; ++j) {
-                        if (g.b_mn) tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, n0 + j * TC_BOX, k0, tc.c);
-                        else        tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, k0, n0 + j * TC_BOX, tc.c);
+                    #pragma unroll
+                    for (int j = 0; j < CTA_N / TC_BOX; ++j) {
+                        if (b_mn) tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, n0 + j * TC_BOX, k0, tc.c);
+                        else      tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, k0, n0 + j * TC_BOX, tc.c);
                     }
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            // stay until the tensor cores have released every stage: the commits arrive on this CTA's barriers
+            for (int s = 0; s < TC_STAGES && ok; ++s) {
+                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
+                if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+            }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
-            const uint32_t a_kstep = g.a_mn ? (2048u >> 4) : (32u >> 4);
-            const uint32_t b_kstep = g.b_mn ? (2048u >> 4) : (32u >> 4);
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            for (int t = pair; t < total_tiles && ok; t += num_pairs) {
                 const TileCoord tc = decode_tile(g, t);
-                const uint32_t idesc = instr_desc(tc.nw, g.a_mn, g.b_mn);
                 if (!(ok = mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, status, 2))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * TC_BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, status, 3))) break;
                     tc_fence_after();
+                    const int k0 = kb * TC_BK;
+                    const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
+                    const int b_mn = g.b_sym ? fetch_transposed(1, tc.tn, k0) : g.b_mn;
+                    // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
+                    const uint32_t a_kstep = a_mn ? (2048u >> 4) : (32u >> 4);
+                    const uint32_t b_kstep = b_mn ? (2048u >> 4) : (32u >> 4);
+                    const uint32_t idesc = instr_desc(a_mn, b_mn);
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-                    const uint64_t da = smem_desc(sa, g.a_mn), db = smem_desc(sb, g.b_mn);
+                    const uint64_t da = smem_desc(sa, a_mn), db = smem_desc(sb, b_mn);
                     #pragma unroll
                     for (int k = 0; k < TC_BK / 16; ++k)
                         tc_mma_bf16(d_tmem, da + (uint64_t)(k * a_kstep), db + (uint64_t)(k * b_kstep), idesc,
                                     (kb | k) != 0 ? 1u : 0u);
-                    tc_commit(bar_empty + 8 * stage);          // frees the stage when these MMAs have read it
+                    tc_commit_pair(bar_empty + 8 * stage);     // frees the stage in both CTAs when these MMAs have read it
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                tc_commit(bar_acc_full + 8 * acc);             // accumulator complete
+                tc_commit_pair(bar_acc_full + 8 * acc);        // accumulator complete, both CTAs' epilogues may read
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
     } else {
-        // ---------------- epilogue (warps 2..9) ----------------
-        // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4); the two warps
-        // of a quadrant take alternate 32-column chunks.  Two chunks are in flight per warp so that the
-        // tensor-memory load of one overlaps the arithmetic and stores of the other.
+        // ---------------- epilogue (warps 2..9, both CTAs) ----------------
+        // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4).  A tile is
+        // written in phases of 128 columns; in a phase the two warps of a quadrant take 64 columns each,
+        // i.e. one 64 x 64 store box column.
         const int quad = warp & 3;
         const int half = (warp - 2) >> 2;
-        const int row_in_tile = quad * 32 + lane;
+        const int row_in_cta = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        uint32_t acc = 0, acc_phase = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) {
+        const bool issuer = threadIdx.x == 64;                 // first epilogue thread: issues and retires TMA stores
+        const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
+        // position of this thread's row inside the staging buffer: box (row half, column half), 128-byte rows
+        const uint32_t box_row = (uint32_t)(row_in_cta & 63);
+        const uint32_t stage_off = (uint32_t)(((row_in_cta >> 6) * 2 + half)) * BOX_BYTES + box_row * 128u;
+        const uint32_t swz = box_row & 7u;
+        uint32_t acc = 0, acc_phase = 0, epi_it = 0;
+        for (int t = pair; t < total_tiles; t += num_pairs) {
             const TileCoord tc = decode_tile(g, t);
-            const int gr = tc.tm * TC_BM + row_in_tile;
+            const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
             const int n0 = tc.tn * TC_BN;
+            const int gr = m0 + row_in_cta;
             const bool row_ok = gr < g.M;
-            const long long mat_off = (long long)tc.c * g.mat_stride;
-            const long long row_off = mat_off + (long long)gr * g.ld;
+            const long long row_off = (long long)tc.c * g.mat_stride + (long long)gr * g.ld;
             float post = 1.0f;
-            if (g.post_mode) { float sc = g.inv_norm[tc.c]; post = g.post_mode == 2 ? sc * sc : sc; }
-            const float c1 = g.c1, c2 = g.c2 * post;
-            const int nchunks = tc.nw >> 5;
-            // operand of the axpy term for the first pair of chunks, requested before the accumulator is ready
-            uint4 cin_raw[2][4];
-            auto load_cin = [&](int ch, uint4* dst) {
-                const int gc0 = n0 + ch * 32;
+            if (g.post_mode) { const float sc = g.inv_norm[tc.c]; post = g.post_mode == 2 ? sc * sc : sc; }
+            const float c1 = g.c1 * post, c2 = g.c2 * post;
+            const int nphases = (g.N - n0 > EPI_COLS) ? 2 : 1;
+            // operand of the axpy term, requested before the accumulator is ready
+            uint4 cin_raw[8];
+            auto load_cin = [&](int ph) {
+                const int gc0 = n0 + ph * EPI_COLS + half * 64;
                 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (row_ok && ch < nchunks && gc0 + 8 * q < g.N) dst[q] = *reinterpret_cast<const uint4*>(g.cin + row_off + gc0 + 8 * q);
-                    else dst[q] = make_uint4(0u, 0u, 0u, 0u);
+                for (int q = 0; q < 8; ++q) {
+                    if (row_ok && gc0 + 8 * q < g.N) cin_raw[q] = *reinterpret_cast<const uint4*>(g.cin + row_off + gc0 + 8 * q);
+                    else cin_raw[q] = make_uint4(0u, 0u, 0u, 0u);
                 }
             };
-            if (g.cin) { load_cin(half, cin_raw[0]); load_cin(half + 2, cin_raw[1]); }
+            if (g.cin) load_cin(0);
             bool ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, status, 4);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = epi_bar_all(3, ok);           // all epilogue threads take the same exit, so no one is left at a barrier
             if (!ok) break;
             tc_fence_after();
-            const uint32_t t_base = tmem_base + lane_base + acc * TC_BN;
-            for (int ch0 = half; ch0 < nchunks; ch0 += 4) {
-                const int ch1 = ch0 + 2;
-                float v[2][32];
-                tmem_ld32(t_base + ch0 * 32, v[0]);
-                if (ch1 < nchunks) tmem_ld32(t_base + ch1 * 32, v[1]);
+            const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
+            for (int ph = 0; ph < nphases; ++ph) {
+                float v[64];
+                tmem_ld32(t_base + ph * EPI_COLS, v);
+                tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
                 tmem_ld_wait();
-                #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int ch = u == 0 ? ch0 : ch1;
-                    const int gc0 = n0 + ch * 32;
-                    if (ch < nchunks && row_ok && gc0 < g.N) {
-                        float* vv = v[u];
-                        if (g.cin) {
-                            const uint32_t w[16] = {cin_raw[u][0].x, cin_raw[u][0].y, cin_raw[u][0].z, cin_raw[u][0].w,
-                                                    cin_raw[u][1].x, cin_raw[u][1].y, cin_raw[u][1].z, cin_raw[u][1].w,
-                                                    cin_raw[u][2].x, cin_raw[u][2].y, cin_raw[u][2].z, cin_raw[u][2].w,
-                                                    cin_raw[u][3].x, cin_raw[u][3].y, cin_raw[u][3].z, cin_raw[u][3].w};
-                            #pragma unroll
-                            for (int h = 0; h < 16; ++h) {
-                                vv[2 * h] = fmaf(c1 * post, __uint_as_float(w[h] << 16), c2 * vv[2 * h]);
-                                vv[2 * h + 1] = fmaf(c1 * post, __uint_as_float(w[h] & 0xffff0000u), c2 * vv[2 * h + 1]);
-                            }
-                        } else {
-                            #pragma unroll
-                            for (int j = 0; j < 32; ++j) vv[j] *= c2;
-                        }
-                        if (g.diag_add != 0.f && gr >= gc0 && gr < gc0 + 32) {
-                            #pragma unroll
-                            for (int j = 0; j < 32; ++j) vv[j] += (gc0 + j == gr) ? g.diag_add : 0.f;
-                        }
-                        #pragma unroll
-                        for (int q = 0; q < 4; ++q)
-                            if (gc0 + 8 * q < g.N) *reinterpret_cast<uint4*>(g.out + row_off + gc0 + 8 * q) = pack8(vv + 8 * q);
-                        if (g.symmetric && (gc0 / TC_BM) < tc.tm) {
-                            // strictly-lower 128-block: the transposed block is not computed anywhere, write it here
-                            __nv_bfloat16* col = g.out + mat_off + (long long)gc0 * g.ld + gr;
-                            #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (gc0 + j < g.N) col[(long long)j * g.ld] = __float2bfloat16_rn(vv[j]);
-                        }
-                    }
+                if (ph == nphases - 1) {
+                    // this warp has read all it needs from the accumulator: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8 * acc);
                 }
-                if (g.cin && ch0 + 4 < nchunks) { load_cin(ch0 + 4, cin_raw[0]); load_cin(ch0 + 6, cin_raw[1]); }
+                const int gc0 = n0 + ph * EPI_COLS + half * 64;
+                if (g.cin) {
+                    const uint32_t w[32] = {cin_raw[0].x, cin_raw[0].y, cin_raw[0].z, cin_raw[0].w, cin_raw[1].x, cin_raw[1].y,
+                                            cin_raw[1].z, cin_raw[1].w, cin_raw[2].x, cin_raw[2].y, cin_raw[2].z, cin_raw[2].w,
+                                            cin_raw[3].x, cin_raw[3].y, cin_raw[3].z, cin_raw[3].w, cin_raw[4].x, cin_raw[4].y,
+                                            cin_raw[4].z, cin_raw[4].w, cin_raw[5].x, cin_raw[5].y, cin_raw[5].z, cin_raw[5].w,
+                                            cin_raw[6].x, cin_raw[6].y, cin_raw[6].z, cin_raw[6].w, cin_raw[7].x, cin_raw[7].y,
+                                            cin_raw[7].z, cin_raw[7].w};
+                    #pragma unroll
+                    for (int h = 0; h < 32; ++h) {
+                        v[2 * h] = fmaf(c1, __uint_as_float(w[h] << 16), c2 * v[2 * h]);
+                        v[2 * h + 1] = fmaf(c1, __uint_as_float(w[h] & 0xffff0000u), c2 * v[2 * h + 1]);
+                    }
+                    if (ph + 1 < nphases) load_cin(ph + 1);
+                } else {
+                    #pragma unroll
+                    for (int j = 0; j < 64; ++j) v[j] *= c2;
+                }
+                if (g.diag_add != 0.f && gr >= gc0 && gr < gc0 + 64) {
+                    #pragma unroll
+                    for (int j = 0; j < 64; ++j) v[j] += (gc0 + j == gr) ? g.diag_add : 0.f;
+                }
+                // the staging buffer is free once the stores issued TC_EPI_BUFS phases ago have read it
+                const uint32_t buf = epi_base + (epi_it % TC_EPI_BUFS) * EPI_BUF_BYTES;
+                if (issuer) bulk_wait_read<TC_EPI_BUFS - 1>();
+                epi_bar_sync(1);
+                #pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const uint4 pk = pack8(v + 8 * q);
+                    const uint32_t addr = buf + stage_off + (((uint32_t)q ^ swz) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk.x), "r"(pk.y), "r"(pk.z), "r"(pk.w)
+                                 : "memory");
+                }
+                fence_proxy_async();           // generic-proxy writes above must be visible to the TMA engine
+                epi_bar_sync(2);
+                if (issuer) {
+                    #pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const int x = n0 + ph * EPI_COLS + (b & 1) * TC_BOX, y = m0 + (b >> 1) * TC_BOX;
+                        if (x < g.N && y < g.M) tma_store_3d(&tma_d, buf + b * BOX_BYTES, x, y, tc.c);   // clipped at the extents
+                    }
+                    bulk_commit();
+                }
+                ++epi_it;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (issuer) bulk_wait_all();           // shared memory must outlive the stores that read it
     }
 
     if (*abort_flag) __nanosleep(200000);      // let copies that are still in flight land before the CTA goes away
     tc_fence_before();
     __syncthreads();
+    cluster_sync();                            // neither CTA leaves (or frees tensor memory) while its peer may still signal it
     tc_fence_after();
     if (warp == 1) {
         __syncwarp();
@@ -378,38 +481,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
 void tc_gemm_plan(TcGemm& g) {
     g.tiles_m = (g.M + TC_BM - 1) / TC_BM;
     g.tiles_n = (g.N + TC_BN - 1) / TC_BN;
-    if (g.symmetric) {
-        int pairs = g.tiles_m / 2;
-        g.tiles_per_mat = pairs * (pairs + 1) + ((g.tiles_m & 1) ? pairs + 1 : 0);
-    } else {
-        g.tiles_per_mat = g.tiles_m * g.tiles_n;
-    }
+    g.tiles_per_mat = g.symmetric ? g.tiles_m * (g.tiles_m + 1) / 2 : g.tiles_m * g.tiles_n;
 }
 
 double tc_gemm_executed_flops(const TcGemm& g) {
     const double kpad = (double)((g.K + TC_BK - 1) / TC_BK * TC_BK);
-    double cols = 0.0;   // sum over tiles of the issued MMA width
-    for (int tm = 0; tm < g.tiles_m; ++tm) {
-        int ntiles = g.symmetric ? tm / 2 + 1 : g.tiles_n;
-        for (int tn = 0; tn < ntiles; ++tn) {
-            int n_left = (g.symmetric ? (g.N < TC_BM * (tm + 1) ? g.N : TC_BM * (tm + 1)) : g.N) - tn * TC_BN;
-            int nw = (n_left + TC_BOX - 1) / TC_BOX * TC_BOX;
-            cols += nw < TC_BN ? nw : TC_BN;
-        }
-    }
-    return 2.0 * TC_BM * cols * kpad * g.C;
+    return 2.0 * TC_BM * TC_BN * kpad * (double)g.tiles_per_mat * g.C;
 }
 
-cudaError_t tc_gemm_configure() {
-    return cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL);
+cudaError_t tc_gemm_configure(int* max_pairs) {
+    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms / 2 * 2));
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = SMEM_TOTAL;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, tc_gemm_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    if (clusters < 1) return cudaErrorInvalidConfiguration;
+    *max_pairs = clusters < sms / 2 ? clusters : sms / 2;
+    return cudaSuccess;
 }
 
-cudaError_t launch_tc_gemm(const CUtensorMap& tma_a, const CUtensorMap& tma_b, const TcGemm& g, int num_sms,
-                           DeviceStatus* status, cudaStream_t stream) {
+cudaError_t launch_tc_gemm(const CUtensorMap& tma_a, const CUtensorMap& tma_b, const CUtensorMap& tma_d,
+                           const TcGemm& g, int max_pairs, DeviceStatus* status, cudaStream_t stream) {
     const int total = g.C * g.tiles_per_mat;
     if (total <= 0) return cudaSuccess;
-    const int grid = total < num_sms ? total : num_sms;
-    tc_gemm_kernel<<<grid, TC_THREADS, SMEM_TOTAL, stream>>>(tma_a, tma_b, g, status);
+    const int pairs = total < max_pairs ? total : max_pairs;
+    tc_gemm_kernel<<<2 * pairs, TC_THREADS, SMEM_TOTAL, stream>>>(tma_a, tma_b, tma_d, g, status);
     return cudaGetLastError();
 }
 

@@ -10,6 +10,7 @@ import paper_2605_26842_b200 as pkg
 from paper_2605_26842_b200 import build as build_mod
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+DEFAULT_CHUNK_BUDGET = 768 << 20     # the library's built-in default; tests that change the knob put it back
 
 
 @pytest.fixture(scope="module")
@@ -44,20 +45,28 @@ def test_query_sizes_state_is_three_fp32_per_parameter(L):
     n = 2 * 64 * 768 * 2048 + 32 * 1024
     assert 12 * n <= sb <= 12 * n + 3 * 256
     assert wb > 0
-    # same shapes in one bucket: two descriptors of one shape need the workspace of one
-    sb2, wb2 = pkg.query_sizes([d[0], d[0]])
-    assert wb2 == pkg.query_sizes([d[0]])[1] and sb2 == 2 * pkg.query_sizes([d[0]])[0]
+    # same shapes share one bucket: once the chunk is bounded by the budget (not by the matrix count),
+    # two descriptors of one shape need the workspace of one
+    pkg.set_chunk_budget(64 << 20)
+    try:
+        sb2, wb2 = pkg.query_sizes([d[0], d[0]])
+        assert wb2 == pkg.query_sizes([d[0]])[1] and sb2 == 2 * pkg.query_sizes([d[0]])[0]
+    finally:
+        pkg.set_chunk_budget(DEFAULT_CHUNK_BUDGET)
 
 
 def test_chunk_budget_changes_workspace(L):
     d = [pkg.MatrixDesc(512, 1024, 32, 0, 0, 0)]
-    pkg.set_chunk_budget(8 << 20)
-    small = pkg.query_sizes(d)[1]
-    pkg.set_chunk_budget(48 << 20)
-    big = pkg.query_sizes(d)[1]
-    assert small < big
-    with pytest.raises(pkg.MonaError):
-        pkg.set_chunk_budget(1000)
+    try:
+        pkg.set_chunk_budget(8 << 20)
+        small = pkg.query_sizes(d)[1]
+        pkg.set_chunk_budget(48 << 20)
+        big = pkg.query_sizes(d)[1]
+        assert small < big
+        with pytest.raises(pkg.MonaError):
+            pkg.set_chunk_budget(1000)
+    finally:
+        pkg.set_chunk_budget(DEFAULT_CHUNK_BUDGET)
 
 
 @pytest.mark.parametrize("desc,status", [
