@@ -346,13 +346,13 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                     for (int t = 0; t < T; ++t) {
                         const int cur = t & 1, nxt = cur ^ 1;
                         TcGemm g1{};     // A = X X^T (wide) or X^T X (tall): lower-triangle tiles only
-                        g1.C = C; g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_mn = g1.b_mn = b.tall ? 1 : 0; g1.symmetric = 1;
+                        g1.C = C; g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_mn = g1.b_mn = b.tall ? 1 : 0; g1.symmetric = 1; g1.ab_same = 1;
                         g1.cin = nullptr; g1.c1 = 0.f; g1.c2 = 1.f;
                         g1.inv_norm = inv_norm; g1.post_mode = t == 0 ? 2 : 0;
                         tc_gemm_plan(g1);
                         MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_x[cur], b.tm_a, g1, h->max_pairs, dstatus, stream));
                         TcGemm g2{};     // B' = b A + c A A + a I, operands and result lower-block-stored
-                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1;
+                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
                         g2.cin = ab; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
                         g2.inv_norm = inv_norm; g2.post_mode = 0; g2.diag_add = ns_a;
                         tc_gemm_plan(g2);

@@ -24,8 +24,14 @@ namespace mona {
 
 namespace {
 
-constexpr int TC_STAGES = 5;
-constexpr int TC_EPI_BUFS = 2;
+#ifndef MONA_TC_STAGES
+#define MONA_TC_STAGES 5
+#endif
+#ifndef MONA_TC_EPI_BUFS
+#define MONA_TC_EPI_BUFS 2
+#endif
+constexpr int TC_STAGES = MONA_TC_STAGES;       // operand ring depth
+constexpr int TC_EPI_BUFS = MONA_TC_EPI_BUFS;   // staging buffers of the store epilogue
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
 constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
@@ -300,12 +306,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                 const TileCoord tc = decode_tile(g, t);
                 const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;      // this CTA's rows of the A operand
                 const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand
+                // diagonal tile of X X^T or A A: both operands are the same rows, staged once
+                const bool shared_ab = g.ab_same && tc.tm == tc.tn;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1))) break;
                     const uint32_t full = full_leader + 8 * stage;
                     const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const int k0 = kb * TC_BK;
-                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, STAGE_TX_BYTES);
+                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, shared_ab ? STAGE_TX_BYTES / 2 : STAGE_TX_BYTES);
                     const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
                     const int b_mn = g.b_sym ? fetch_transposed(1, tc.tn, k0) : g.b_mn;
                     #pragma unroll
@@ -313,10 +321,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                         if (a_mn) tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, m0 + j * TC_BOX, k0, tc.c);
                         else      tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, k0, m0 + j * TC_BOX, tc.c);
                     }
-                    #pragma unroll
-                    for (int j = 0; j < CTA_N / TC_BOX; ++j) {
-                        if (b_mn) tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, n0 + j * TC_BOX, k0, tc.c);
-                        else      tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, k0, n0 + j * TC_BOX, tc.c);
+                    if (!shared_ab) {
+                        #pragma unroll
+                        for (int j = 0; j < CTA_N / TC_BOX; ++j) {
+                            if (b_mn) tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, n0 + j * TC_BOX, k0, tc.c);
+                            else      tma_load_3d(sb + j * BOX_BYTES, &tma_b, full, k0, n0 + j * TC_BOX, tc.c);
+                        }
                     }
                     if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -337,17 +347,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                 if (!(ok = mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, status, 2))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * TC_BN;
+                const bool shared_ab = g.ab_same && tc.tm == tc.tn;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, status, 3))) break;
                     tc_fence_after();
                     const int k0 = kb * TC_BK;
                     const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
-                    const int b_mn = g.b_sym ? fetch_transposed(1, tc.tn, k0) : g.b_mn;
+                    const int b_mn = shared_ab ? a_mn : (g.b_sym ? fetch_transposed(1, tc.tn, k0) : g.b_mn);
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
                     const uint32_t a_kstep = a_mn ? (2048u >> 4) : (32u >> 4);
                     const uint32_t b_kstep = b_mn ? (2048u >> 4) : (32u >> 4);
                     const uint32_t idesc = instr_desc(a_mn, b_mn);
-                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    const uint32_t sa = base + stage * STAGE_BYTES, sb = shared_ab ? sa : sa + A_STAGE_BYTES;
                     const uint64_t da = smem_desc(sa, a_mn), db = smem_desc(sb, b_mn);
                     #pragma unroll
                     for (int k = 0; k < TC_BK / 16; ++k)

@@ -28,6 +28,8 @@ struct TcGemm {
     int a_mn, b_mn;             // 1: operand is MN-major (ignored for an operand flagged *_sym)
     int a_sym, b_sym;           // 1: operand is a symmetric matrix stored as its lower block triangle
     int symmetric;              // 1: D = D^T, compute lower-triangle tiles only
+    int ab_same;                // 1: both operands are the same tensor in the same form (X X^T, A A): a diagonal
+                                //    tile stages its operand rows once and uses them on both sides
     int tiles_m, tiles_n, tiles_per_mat;
     const __nv_bfloat16* cin;   // may be null; when D is symmetric, Cin is lower-block-stored like D
     long long ld, mat_stride;   // leading dimension and per-matrix stride of cin, in elements
