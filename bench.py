@@ -94,9 +94,10 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(wl, per_shape: int = 1):
-    """Times the fp64 oracle, as it stands, on `per_shape` matrices of every distinct shape of the
-    workload (one full step each) and extrapolates to the whole set.  Returns (steps/s, description, threads)."""
+def oracle_sample(wl, budget_s: float = 12.0):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: one full step on matrices of
+    every distinct shape, repeated round-robin over the shapes until about `budget_s` seconds of CPU work
+    are spent, then extrapolated to the whole set by matrix count.  Returns (steps/s, description, threads)."""
     import numpy as np
     import oracle.mona_oracle as orc
     try:
@@ -109,21 +110,27 @@ def oracle_sample(wl, per_shape: int = 1):
         counts[(s.rows, s.cols)] = counts.get((s.rows, s.cols), 0) + s.batch
     rng = np.random.default_rng(wl.seed)
     hp = orc.Hyper(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha)
-    total, parts, spent = 0.0, [], 0.0
-    for (m, n), cnt in counts.items():
-        ts = []
-        for _ in range(per_shape):
+    times = {k: [] for k in counts}
+    spent = 0.0
+    while True:
+        for (m, n) in counts:
             W = rng.standard_normal((m, n)) * 0.02
             G = rng.standard_normal((m, n)) * wl.sigma
             st = orc.OracleState(m, n)
             t0 = time.perf_counter()
             orc.mona_step(W, G, st, hp)
-            ts.append(time.perf_counter() - t0)
-        t = sum(ts) / len(ts)
-        spent += sum(ts)
+            dt = time.perf_counter() - t0
+            times[(m, n)].append(dt)
+            spent += dt
+        if spent >= budget_s or len(next(iter(times.values()))) >= 64:
+            break
+    total, parts = 0.0, []
+    for (m, n), cnt in counts.items():
+        t = sum(times[(m, n)]) / len(times[(m, n)])
         total += cnt * t
         parts.append(f"{m}x{n}: {t * 1e3:.1f} ms x {cnt}")
-    desc = (f"fp64 numpy oracle, {per_shape} matrix per distinct shape, one full step each ({spent:.1f} s of CPU work), "
+    reps = len(next(iter(times.values())))
+    desc = (f"fp64 numpy oracle, {reps} matrices of every distinct shape, one full step each ({spent:.1f} s of CPU work), "
             f"extrapolated by matrix count: " + "; ".join(parts))
     return 1.0 / total, desc, threads
 
@@ -156,7 +163,7 @@ def run_reference(args):
     desc = ""
     threads = 1
     for i in range(args.warmup + args.steps):
-        v, desc, threads = oracle_sample(wl, 1)
+        v, desc, threads = oracle_sample(wl, 10.0)
         if i >= args.warmup:
             vals.append(v)
     value = len(vals) / sum(1.0 / v for v in vals)
@@ -324,7 +331,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        v, desc, threads = oracle_sample(wl, 1)
+        v, desc, threads = oracle_sample(wl, 15.0)
         cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
     if rank == 0:
