@@ -186,7 +186,8 @@ def main():
     ap.add_argument("--impl", default="mona", choices=["mona", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--chunk-mb", type=int, default=None, help="override the L2 chunk budget (MiB)")
+    ap.add_argument("--chunk-mb", type=int, default=None, help="override the chunk budget (MiB)")
+    ap.add_argument("--no-overlap", action="store_true", help="keep all chunks on one stream")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -207,6 +208,8 @@ def main():
     dev = torch.device("cuda", local_rank)
     if args.chunk_mb:
         pkg.set_chunk_budget(args.chunk_mb << 20)
+    if args.no_overlap:
+        pkg.set_chunk_overlap(False)
 
     free_bytes, _ = torch.cuda.mem_get_info(dev)
     wl, fit_note = pick_workload(args.config, args.layers, free_bytes)

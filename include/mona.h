@@ -95,6 +95,12 @@ mona_status mona_default_hparams(mona_hparams* hp);
  * mona_query_sizes() and mona_create() only. */
 mona_status mona_set_chunk_budget(size_t bytes);
 
+/* Tuning knob, process-wide: 1 (default) pipelines consecutive chunks over two streams - the caller's and
+ * one the handle owns, joined by events before mona_step*() returns to the caller's stream - so that the
+ * partial last wave and the launch gap of one chunk's kernels are filled by the other chunk's; 0 keeps
+ * every launch on the caller's stream.  Results are identical either way; the workspace holds two chunks. */
+mona_status mona_set_chunk_overlap(int enabled);
+
 /* Bytes the caller must provide for the optimizer state (M, A, G_prev: 3 fp32 per parameter,
  * Algorithm 1 line 1) and for the Newton-Schulz workspace.  Host only; no device is touched. */
 mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc,

@@ -49,6 +49,7 @@ def lib() -> C.CDLL:
     vp, vpp = C.c_void_p, C.POINTER(C.c_void_p)
     L.mona_default_hparams.argtypes = [C.POINTER(Hparams)]
     L.mona_set_chunk_budget.argtypes = [C.c_size_t]
+    L.mona_set_chunk_overlap.argtypes = [C.c_int]
     L.mona_query_sizes.argtypes = [C.POINTER(MatrixDesc), C.c_int64, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.mona_create.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_step.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vp]
@@ -63,7 +64,7 @@ def lib() -> C.CDLL:
     L.mona_last_error.restype = C.c_char_p
     L.mona_destroy.argtypes = [vp]
     L.mona_destroy.restype = None
-    for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_query_sizes", "mona_create", "mona_step",
+    for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_set_chunk_overlap", "mona_query_sizes", "mona_create", "mona_step",
                  "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops"):
         getattr(L, name).restype = C.c_int
     _lib = L
@@ -86,6 +87,12 @@ def set_chunk_budget(nbytes: int) -> None:
     st = lib().mona_set_chunk_budget(nbytes)
     if st:
         raise MonaError(st, "chunk budget must be at least 1 MiB")
+
+
+def set_chunk_overlap(enabled: bool) -> None:
+    st = lib().mona_set_chunk_overlap(1 if enabled else 0)
+    if st:
+        raise MonaError(st, "mona_set_chunk_overlap")
 
 
 def _desc_array(descs: Sequence[MatrixDesc]):

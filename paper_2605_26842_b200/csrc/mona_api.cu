@@ -25,12 +25,22 @@ using namespace mona;
 namespace {
 
 // ---- workspace layout -------------------------------------------------------------------------------
+// [status word | control block of slot 0 | control block of slot 1 | iterates of slot 0 | iterates of slot 1]
+// Consecutive chunks alternate between two slots (and two streams), so that the last wave of each GEMM
+// launch is filled by the other chunk's tiles and launch gaps of one chunk are covered by the other.
+constexpr int NSLOTS = 2;
 constexpr size_t WS_STATUS_OFF = 0;
-constexpr size_t WS_COUNTERS_OFF = 256;
-constexpr size_t WS_INVNORM_OFF = 2048;
-constexpr size_t WS_PARTIALS_OFF = 4096;
-constexpr size_t WS_DATA_OFF = 256 * 1024;
-static_assert(WS_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS <= WS_DATA_OFF, "control block overflow");
+constexpr size_t WS_CTRL_OFF = 4096;                 // first control block
+constexpr size_t WS_CTRL_BYTES = 256 * 1024;         // per slot
+constexpr size_t CTRL_COUNTERS_OFF = 0;
+constexpr size_t CTRL_INVNORM_OFF = 2048;
+constexpr size_t CTRL_PARTIALS_OFF = 4096;
+constexpr size_t WS_DATA_OFF = WS_CTRL_OFF + NSLOTS * WS_CTRL_BYTES;
+static_assert(CTRL_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS <= WS_CTRL_BYTES, "control block overflow");
+static_assert(sizeof(unsigned int) * MAXC <= CTRL_INVNORM_OFF && sizeof(float) * MAXC <= CTRL_PARTIALS_OFF - CTRL_INVNORM_OFF, "control block overflow");
+
+// 1: consecutive chunks are pipelined over two streams; 0: everything runs on the caller's stream.
+int g_chunk_overlap = 1;
 
 // Bytes of bf16 iterates (X_t, X_{t+1}, A_t, B_t) a chunk may hold so that it stays resident in L2
 // between the 3T GEMMs of the iteration.
@@ -52,10 +62,10 @@ struct Bucket {
     int Cb = 1, Cf = 1;         // chunk capacity: bf16 tensor-core mode / fp32 mode
     int slabs = 1;
     int64_t slab_len = 0;
-    size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;          // bf16 mode, bytes from workspace base
+    size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;          // bf16 mode, bytes from the slot's iterate base
     size_t off32_x[2] = {0, 0}, off32_a = 0, off32_b = 0;    // fp32 mode
     size_t data_bytes = 0;
-    CUtensorMap tm_x[2], tm_a, tm_b;
+    CUtensorMap tm_x[NSLOTS][2], tm_a[NSLOTS], tm_b[NSLOTS];
 };
 
 struct Plan {
@@ -64,7 +74,7 @@ struct Plan {
     std::vector<int> desc_bucket;          // bucket of descriptor i
     std::vector<int64_t> desc_pos;         // position of descriptor i's matrix 0 inside its bucket
     std::vector<int64_t> desc_first_gid;   // global matrix index (descriptor order) of matrix 0
-    size_t state_bytes = 0, workspace_bytes = 0;
+    size_t state_bytes = 0, workspace_bytes = 0, slot_bytes = 0;
 };
 
 mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan, std::string& err) {
@@ -120,11 +130,11 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         cb = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(cb, MAXC), count));
         b.Cb = (int)cb;
         b.Cf = (int)std::max<int64_t>(1, cb / 2);
-        size_t off = WS_DATA_OFF;
+        size_t off = 0;
         for (int i = 0; i < 2; ++i) { b.off_x[i] = off; off += align_up((size_t)b.Cb * b.e * 2, 1024); }
         b.off_a = off; off += align_up((size_t)b.Cb * b.s * b.s * 2, 1024);
         b.off_b = off; off += align_up((size_t)b.Cb * b.s * b.s * 2, 1024);
-        size_t off32 = WS_DATA_OFF;
+        size_t off32 = 0;
         for (int i = 0; i < 2; ++i) { b.off32_x[i] = off32; off32 += align_up((size_t)b.Cf * b.e * 4, 1024); }
         b.off32_a = off32; off32 += align_up((size_t)b.Cf * b.s * b.s * 4, 1024);
         b.off32_b = off32; off32 += align_up((size_t)b.Cf * b.s * b.s * 4, 1024);
@@ -132,7 +142,8 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         max_data = std::max(max_data, b.data_bytes);
     }
     plan.state_bytes = (size_t)state_floats * 4;
-    plan.workspace_bytes = max_data;
+    plan.slot_bytes = align_up(max_data, 1024);
+    plan.workspace_bytes = WS_DATA_OFF + NSLOTS * plan.slot_bytes;
     return MONA_OK;
 }
 
@@ -206,6 +217,11 @@ mona_status mona_set_chunk_budget(size_t bytes) {
     return MONA_OK;
 }
 
+mona_status mona_set_chunk_overlap(int enabled) {
+    g_chunk_overlap = enabled ? 1 : 0;
+    return MONA_OK;
+}
+
 mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc, size_t* state_bytes, size_t* workspace_bytes) {
     Plan plan;
     std::string err;
@@ -248,9 +264,12 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
     for (Bucket& b : h->plan.buckets) {
         if (!b.tc_ok) continue;
         bool ok = true;
-        for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.tm_x[i], h->ws + b.off_x[i], b.cols, b.rows, b.Cb);
-        ok = ok && encode_map(encode, &b.tm_a, h->ws + b.off_a, b.s, b.s, b.Cb);
-        ok = ok && encode_map(encode, &b.tm_b, h->ws + b.off_b, b.s, b.s, b.Cb);
+        for (int sl = 0; sl < NSLOTS; ++sl) {
+            uint8_t* data = h->ws + WS_DATA_OFF + sl * h->plan.slot_bytes;
+            for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.tm_x[sl][i], data + b.off_x[i], b.cols, b.rows, b.Cb);
+            ok = ok && encode_map(encode, &b.tm_a[sl], data + b.off_a, b.s, b.s, b.Cb);
+            ok = ok && encode_map(encode, &b.tm_b[sl], data + b.off_b, b.s, b.s, b.Cb);
+        }
         if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
     }
     MONA_CUDA(h, tc_gemm_configure(&h->max_pairs));
@@ -281,7 +300,6 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
         if (((uintptr_t)params[i] & 15) || ((uintptr_t)grads[i] & 15) || (o_out && o_out[i] && ((uintptr_t)o_out[i] & 15)))
             return h->fail(MONA_ERR_ALIGNMENT, "descriptor %lld: pointers must be 16-byte aligned", (long long)i);
     }
-    cudaStream_t stream = (cudaStream_t)stream_v;
     MONA_CUDA(h, cudaSetDevice(h->device));
 
     PrologueScalars ps;
@@ -295,9 +313,20 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
     const float ns_a = (float)hp->ns_a, ns_b = (float)hp->ns_b, ns_c = (float)hp->ns_c;
 
     DeviceStatus* dstatus = (DeviceStatus*)(h->ws + WS_STATUS_OFF);
-    unsigned int* counters = (unsigned int*)(h->ws + WS_COUNTERS_OFF);
-    float* inv_norm = (float*)(h->ws + WS_INVNORM_OFF);
-    float* partials = (float*)(h->ws + WS_PARTIALS_OFF);
+    // chunks alternate between the caller's stream (slot 0) and the handle's own stream (slot 1)
+    int64_t total_chunks = 0;
+    for (const Bucket& b : plan.buckets) {
+        const bool tcb = (hp->ns_precision == 0) && b.tc_ok && T >= 1;
+        const int capb = tcb ? b.Cb : b.Cf;
+        total_chunks += ((int64_t)b.mats.size() + capb - 1) / capb;
+    }
+    const bool overlap = g_chunk_overlap && total_chunks > 1;
+    cudaStream_t slot_stream[NSLOTS] = {(cudaStream_t)stream_v, overlap ? h->side : (cudaStream_t)stream_v};
+    if (overlap) {
+        MONA_CUDA(h, cudaEventRecord(h->ev_fork, slot_stream[0]));
+        MONA_CUDA(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+    }
+    int64_t chunk_index = 0;
     h->launches = 0;
     h->flops_exec = 0.0;
     h->flops_dense = 0.0;
@@ -326,14 +355,22 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                 ptrs.o[c] = (o_out && o_out[mr.desc]) ? (float*)o_out[mr.desc] + mr.b * d.batch_stride : nullptr;
                 ptrs.gid[c] = (int)(plan.desc_first_gid[mr.desc] + mr.b);
             }
+            const int slot = overlap ? (int)(chunk_index % NSLOTS) : 0;
+            ++chunk_index;
+            cudaStream_t stream = slot_stream[slot];
+            uint8_t* ctrl = h->ws + WS_CTRL_OFF + slot * WS_CTRL_BYTES;
+            uint8_t* data = h->ws + WS_DATA_OFF + slot * plan.slot_bytes;
+            unsigned int* counters = (unsigned int*)(ctrl + CTRL_COUNTERS_OFF);
+            float* inv_norm = (float*)(ctrl + CTRL_INVNORM_OFF);
+            float* partials = (float*)(ctrl + CTRL_PARTIALS_OFF);
             float* Mc = Mst + start * b.e;
             float* Ac = Ast + start * b.e;
             float* Gc = Gst + start * b.e;
-            __nv_bfloat16* xb[2] = {(__nv_bfloat16*)(h->ws + b.off_x[0]), (__nv_bfloat16*)(h->ws + b.off_x[1])};
-            __nv_bfloat16* ab = (__nv_bfloat16*)(h->ws + b.off_a);
-            float* xf[2] = {(float*)(h->ws + b.off32_x[0]), (float*)(h->ws + b.off32_x[1])};
-            float* af = (float*)(h->ws + b.off32_a);
-            float* bf = (float*)(h->ws + b.off32_b);
+            __nv_bfloat16* xb[2] = {(__nv_bfloat16*)(data + b.off_x[0]), (__nv_bfloat16*)(data + b.off_x[1])};
+            __nv_bfloat16* ab = (__nv_bfloat16*)(data + b.off_a);
+            float* xf[2] = {(float*)(data + b.off32_x[0]), (float*)(data + b.off32_x[1])};
+            float* af = (float*)(data + b.off32_a);
+            float* bf = (float*)(data + b.off32_b);
 
             if (phase_mask & 1u) {
                 MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16, vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
@@ -350,13 +387,13 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                         g1.cin = nullptr; g1.c1 = 0.f; g1.c2 = 1.f;
                         g1.inv_norm = inv_norm; g1.post_mode = t == 0 ? 2 : 0;
                         tc_gemm_plan(g1);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_x[cur], b.tm_a, g1, h->max_pairs, dstatus, stream));
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[slot][cur], b.tm_x[slot][cur], b.tm_a[slot], g1, h->max_pairs, dstatus, stream));
                         TcGemm g2{};     // B' = b A + c A A + a I, operands and result lower-block-stored
                         g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
                         g2.cin = ab; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
                         g2.inv_norm = inv_norm; g2.post_mode = 0; g2.diag_add = ns_a;
                         tc_gemm_plan(g2);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_a, b.tm_a, b.tm_b, g2, h->max_pairs, dstatus, stream));
+                        MONA_CUDA(h, launch_tc_gemm(b.tm_a[slot], b.tm_a[slot], b.tm_b[slot], g2, h->max_pairs, dstatus, stream));
                         TcGemm g3{};
                         g3.C = C; g3.K = (int)b.s; g3.symmetric = 0;
                         g3.cin = nullptr; g3.c1 = 0.f; g3.c2 = 1.f;
@@ -364,11 +401,11 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                         if (!b.tall) {   // X' = B' X : B' is the symmetric "A" operand, X the MN-major "B" operand
                             g3.M = (int)b.s; g3.N = (int)b.l; g3.a_sym = 1; g3.b_mn = 1;
                             tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_b, b.tm_x[cur], b.tm_x[nxt], g3, h->max_pairs, dstatus, stream));
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_b[slot], b.tm_x[slot][cur], b.tm_x[slot][nxt], g3, h->max_pairs, dstatus, stream));
                         } else {         // X' = X B' : X is K-major, the symmetric B' serves as its own transpose
                             g3.M = (int)b.l; g3.N = (int)b.s; g3.a_mn = 0; g3.b_sym = 1;
                             tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[cur], b.tm_b, b.tm_x[nxt], g3, h->max_pairs, dstatus, stream));
+                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[slot][cur], b.tm_b[slot], b.tm_x[slot][nxt], g3, h->max_pairs, dstatus, stream));
                         }
                         h->launches += 3;
                         h->flops_exec += tc_gemm_executed_flops(g1) + tc_gemm_executed_flops(g2) + tc_gemm_executed_flops(g3);
@@ -419,6 +456,10 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                 ++h->launches;
             }
         }
+    }
+    if (overlap) {
+        MONA_CUDA(h, cudaEventRecord(h->ev_join, h->side));
+        MONA_CUDA(h, cudaStreamWaitEvent(slot_stream[0], h->ev_join, 0));
     }
     return MONA_OK;
 }

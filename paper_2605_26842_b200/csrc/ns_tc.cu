@@ -35,6 +35,9 @@ constexpr int TC_EPI_BUFS = MONA_TC_EPI_BUFS;   // staging buffers of the store 
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
 constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
+// 320 threads x 160 registers leave room on the SM for one 256-thread block of the elementwise kernels, so
+// a prologue or update of the neighbouring chunk can run beside a resident GEMM CTA
+constexpr int TC_MAX_REGS = 160;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows staged by one CTA
 constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
@@ -254,7 +257,7 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
     return r;
 }
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(TC_MAX_REGS)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
                const __grid_constant__ CUtensorMap tma_d, TcGemm g, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
