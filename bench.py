@@ -154,10 +154,9 @@ def pick_workload(index, layers, free_bytes):
 
 def run_reference(args):
     """`--impl reference`: the oracle on the host cores, same metric and configuration."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    from paper_2605_26842_b200 import shard, synth
+    if shard.env_rank()[0] != 0:
         return
-    from paper_2605_26842_b200 import synth
     wl = synth.workload(args.config, args.layers)
     vals = []
     desc = ""
@@ -197,9 +196,8 @@ def main():
     import paper_2605_26842_b200 as pkg
     from paper_2605_26842_b200 import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2605_26842_b200 import shard
+    rank, local_rank, world = shard.env_rank()
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -260,13 +258,9 @@ def main():
         raise RuntimeError(f"device status {pkg.STATUS_NAMES[st]} at matrix {bad}")
     launches_per_step = opt.last_launch_count()
     flops_exec, flops_dense = opt.last_ns_flops()
-    total_ms = sum(ms)
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = shard.max_over_ranks(sum(ms), dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = shard.whole_job_rate(1.0, world, ms_per_step * 1e-3)
 
     # ---- per-phase passes (one phase alone; state keeps evolving, which does not change the work) ----
     n_phase = max(2, min(args.steps, 3))
@@ -321,12 +315,8 @@ def main():
                 torch.cuda.synchronize(dev)
                 if i > 0:
                     e_ms.append(e0.elapsed_time(e1))
-            e_total = sum(e_ms)
-            if dist is not None:
-                t = torch.tensor([e_total], dtype=torch.float64, device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e_total = float(t.item())
-            e2e = {"value": world * 1e3 / (e_total / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            e_total = shard.max_over_ranks(sum(e_ms), dist, dev)
+            e2e = {"value": shard.whole_job_rate(1.0, world, e_total / n_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                    "steps": n_e2e, "api": "mona_step_host (pinned host gradients in, updated parameters out)"}
             del g_host, p_host
         except Exception as exc:   # e.g. not enough pinned host memory
