@@ -41,6 +41,8 @@ static_assert(sizeof(unsigned int) * MAXC <= CTRL_INVNORM_OFF && sizeof(float) *
 
 // 1: consecutive chunks are pipelined over two streams; 0: everything runs on the caller's stream.
 int g_chunk_overlap = 1;
+// 1: X' = B' X runs on 256 x 512 macro-tiles.
+int g_wide_g3 = 1;
 
 // Bytes of bf16 iterates (X_t, X_{t+1}, A_t, B_t) a chunk may hold so that it stays resident in L2
 // between the 3T GEMMs of the iteration.
@@ -395,7 +397,7 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                         tc_gemm_plan(g2);
                         MONA_CUDA(h, launch_tc_gemm(b.tm_a[slot], b.tm_a[slot], b.tm_b[slot], g2, h->max_pairs, dstatus, stream));
                         TcGemm g3{};
-                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0;
+                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0; g3.wide = g_wide_g3;
                         g3.cin = nullptr; g3.c1 = 0.f; g3.c2 = 1.f;
                         g3.inv_norm = inv_norm; g3.post_mode = t == 0 ? 1 : 0;
                         if (!b.tall) {   // X' = B' X : B' is the symmetric "A" operand, X the MN-major "B" operand

@@ -30,7 +30,9 @@ struct TcGemm {
     int symmetric;              // 1: D = D^T, compute lower-triangle tiles only
     int ab_same;                // 1: both operands are the same tensor in the same form (X X^T, A A): a diagonal
                                 //    tile stages its operand rows once and uses them on both sides
-    int tiles_m, tiles_n, tiles_per_mat;
+    int wide;                   // 1 (non-symmetric D only): a pair computes 256 x 512 macro-tiles, two tiles that share
+                                //    one staged slice of the A operand, one per tensor-memory accumulator
+    int tiles_m, tiles_n, tiles_per_mat;   // tiles_per_mat counts macro-tiles when `wide`
     const __nv_bfloat16* cin;   // may be null; when D is symmetric, Cin is lower-block-stored like D
     long long ld, mat_stride;   // leading dimension and per-matrix stride of cin, in elements
     float c1, c2;
@@ -39,7 +41,7 @@ struct TcGemm {
     int post_mode;              // 0: post = 1, 1: post = inv, 2: post = inv^2
 };
 
-// Fills the tile counts of `g` from M, N, symmetric.
+// Fills the tile counts of `g` from M, N, symmetric, wide.
 void tc_gemm_plan(TcGemm& g);
 // Tensor-core flops (2*M*N*K per issued MMA, padded extents included) one launch of `g` executes.
 double tc_gemm_executed_flops(const TcGemm& g);
