@@ -29,6 +29,21 @@ if ROOT not in sys.path:
 METRIC = "mona_optimizer_steps_per_s"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the GEMM kernel from the ncu capture
+# summarised in profiles/tc_gemm_kernel_moe7b_768x2048_per_launch.md: mean over the 15 launches of one 93-matrix
+# 768x2048 chunk, the launch shape that makes up most of the default workload.  Valid only for the kernel source
+# the counters were taken with (hash of ns_tc.cu + ns_tc.cuh).
+NCU_TRAFFIC = {"source_sha256_16": "631c532b94439144", "bytes_per_launch": 358.4e6}
+
+
+def kernel_traffic():
+    """DRAM bytes per GEMM launch from the committed ncu capture, or None once the kernel source has changed."""
+    import hashlib
+    try:
+        src = b"".join(open(os.path.join(ROOT, "paper_2605_26842_b200", "csrc", f), "rb").read() for f in ("ns_tc.cu", "ns_tc.cuh"))
+    except OSError:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"] if hashlib.sha256(src).hexdigest()[:16] == NCU_TRAFFIC["source_sha256_16"] else None
 
 
 def load_peaks():
@@ -286,7 +301,8 @@ def main():
                 "frac": ns_tflops / peaks["bf16_tflops_sustained"], "peak_source": peak_src + " (sustained bf16 GEMM)",
                 "frac_of_burst_peak": ns_tflops / peaks["bf16_tflops"], "frac_of_nominal_2250": ns_tflops / 2250.0,
                 "flops_per_launch": flops_exec / max(1, ns_launches), "launches_per_step": ns_launches,
-                "avg_launch_us": ms_ns * 1e3 / max(1, ns_launches), "traffic": None,
+                "avg_launch_us": ms_ns * 1e3 / max(1, ns_launches), "traffic": kernel_traffic(),
+                "traffic_unit": "DRAM bytes per launch (ncu, 93-matrix 768x2048 chunk)",
                 "dense_equivalent_tflops": flops_dense / (ms_ns * 1e-3) / 1e12}
     phases = {"prologue_ms": ms_pro, "prologue_gbs": pro_gbs, "prologue_frac_of_hbm_peak": pro_gbs / peaks["hbm_gbs"],
               "prologue_frac_of_nominal_8000": pro_gbs / 8000.0, "prologue_bytes_per_elem": 12 + g_elem + 14,
