@@ -13,6 +13,8 @@ notation, with no blocking, fusion or reordering:
   * Eq. newton_schulz                       -> newton_schulz(): X_0 = M/||M||_F, quintic iteration
   * gamma = 0.2 sqrt(max(m, n))             -> update_scale()
   * Eq. muon_update                         -> apply_update(): W <- W - eta (gamma O + lambda W)
+  * MONA-Lite (section "Efficient Deployment with Reduced Overhead"): G_{k-1} and A_k kept in
+    bfloat16, equations unchanged          -> round_bf16(), Hyper.state_dtype = "bf16"
 
 Readings taken where the paper is silent (all are arguments, none is hidden):
   * First step: G_0 = 0 (Algorithm 1, line 1), so D_1 = G_1.
@@ -22,6 +24,10 @@ Readings taken where the paper is silent (all are arguments, none is hidden):
   * The iteration is applied to the m x n matrix as written, never transposed.
   * gamma uses max(m, n) of the individual matrix.
   * Weight decay sits inside the eta bracket and uses W_k (the value before the update).
+  * MONA-Lite: the paper only says the two buffers are stored in bfloat16.  Taken here as: A_k is
+    formed in full precision, rounded once (nearest, ties to even) when it is stored, and the stored
+    value is the one G~_k uses, so that the state alone determines the next step; G_{k-1} is the
+    rounded G_k.  M_k and everything downstream stay in full precision.
 
 Every function here is pinned by tests that do not call it to produce their expected value
 (closed forms, scalar hand arithmetic, a library SVD, invariants); nothing is "parity unpinned".
@@ -53,6 +59,7 @@ class Hyper:
     norm_eps: float = 1e-7
     scale_mode: int = 0          # 0: gamma = scale_value * sqrt(max(m, n)); 1: gamma = scale_value
     scale_value: float = 0.2
+    state_dtype: str = "fp32"    # "bf16": MONA-Lite, G_{k-1} and A_k stored in bfloat16
 
 
 class OracleState:
@@ -69,10 +76,25 @@ class OracleState:
         return s
 
 
-def acceleration(G, G_prev, A_prev, beta_a, alpha):
-    """Eq. alto_diff, alto_accel, alto_grad (Algorithm 1, lines 4-6)."""
+def round_bf16(x):
+    """Value of x after storage in bfloat16 (1 sign, 8 exponent, 7 fraction bits): the nearest
+    representable number, ties to the even fraction.  Done on the bit pattern of the float32 value,
+    of which a bfloat16 is the upper half."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    u = u + 0x7FFF + ((u >> 16) & 1)
+    return ((u >> 16) << 16).astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def keep(x):
+    """Full-precision storage."""
+    return x
+
+
+def acceleration(G, G_prev, A_prev, beta_a, alpha, store=keep):
+    """Eq. alto_diff, alto_accel, alto_grad (Algorithm 1, lines 4-6).  `store` is the storage format
+    of A_k (identity, or round_bf16 for MONA-Lite)."""
     D = G - G_prev
-    A = beta_a * A_prev + (1.0 - beta_a) * D
+    A = store(beta_a * A_prev + (1.0 - beta_a) * D)
     G_tilde = G + alpha * A
     return A, G_tilde
 
@@ -112,12 +134,13 @@ def mona_step(W, G, state: OracleState, hp: Hyper):
     Returns (W_next, O) as float64 arrays."""
     W = np.asarray(W, dtype=np.float64)
     G = np.asarray(G, dtype=np.float64)
-    A, G_tilde = acceleration(G, state.G_prev, state.A, hp.accel_beta, hp.accel_alpha)
+    store = round_bf16 if hp.state_dtype == "bf16" else keep
+    A, G_tilde = acceleration(G, state.G_prev, state.A, hp.accel_beta, hp.accel_alpha, store)
     M = momentum(state.M, G_tilde, hp.momentum)
     O = newton_schulz(M, hp.ns_steps, hp.ns_a, hp.ns_b, hp.ns_c, hp.norm_eps)
     gamma = update_scale(W.shape[0], W.shape[1], hp.scale_mode, hp.scale_value)
     W_next = apply_update(W, O, hp.lr, gamma, hp.weight_decay)
     state.A = A
     state.M = M
-    state.G_prev = G.copy()          # Algorithm 1, line 10
+    state.G_prev = store(G.copy())   # Algorithm 1, line 10
     return W_next, O

@@ -7,9 +7,14 @@ iteration of Eq. newton_schulz acts on the singular values only,
     NS_T(M) = U diag(p^T(sigma_i / ||M||_F)) V^T,   p(x) = a x + b x^3 + c x^5,
 which is a closed form, not the matrix iteration the oracle runs.
 
-Usage:  python tests/golden/derive_hand_values.py   (rewrites the three .txt files)
+The MONA-Lite case repeats the diagonal 2x2 steps with A_k and G_{k-1} rounded to bfloat16 when stored.
+The rounding is done here on exact rationals from the definition of the format (8 significant bits,
+nearest, ties to even), not on bit patterns.
+
+Usage:  python tests/golden/derive_hand_values.py   (rewrites the .txt files)
 """
 from decimal import Decimal as D, getcontext
+from fractions import Fraction as F
 import os
 
 import numpy as np
@@ -101,5 +106,46 @@ def write_3x2():
     open(os.path.join(HERE, "hand_3x2.txt"), "w").write("\n".join(lines) + "\n")
 
 
+def bf16(x: F) -> F:
+    """Nearest number with 8 significant binary digits, ties to the even last digit (exact rationals)."""
+    if x == 0:
+        return x
+    sign = -1 if x < 0 else 1
+    x = abs(x)
+    e = 0
+    while F(2) ** (e + 1) <= x:
+        e += 1
+    while F(2) ** e > x:
+        e -= 1
+    unit = F(2) ** (e - 7)              # spacing of 8-bit significands in [2^e, 2^(e+1))
+    q = x / unit
+    lo = q.numerator // q.denominator
+    rem = q - lo
+    if rem > F(1, 2) or (rem == F(1, 2) and lo % 2 == 1):
+        lo += 1
+    return sign * lo * unit
+
+
+def write_lite_2x2():
+    # Lines 4-7 and 10 of Algorithm 1 on diagonal 2x2 matrices with bfloat16 storage of A_k and G_{k-1}:
+    # G_1 = diag(0.3, 3), G_2 = diag(0.3, 4); beta_a = 0.9, alpha = -5, mu = 0.5.
+    beta, alpha, mu = F(9, 10), F(-5), F(1, 2)
+    Gs = [[F(3, 10), F(3)], [F(3, 10), F(4)]]
+    A = [F(0), F(0)]; M = [F(0), F(0)]; Gp = [F(0), F(0)]
+    lines = ["# MONA-Lite (G_{k-1} and A_k stored in bfloat16: nearest, ties to even; exact rational arithmetic otherwise).",
+             "# Two steps of lines 4-7 and 10 of Algorithm 1 on diagonal 2x2 matrices: G_1 = diag(0.3, 3), G_2 = diag(0.3, 4);",
+             "# beta_a=0.9 alpha=-5 mu=0.5.  A is rounded when stored and the stored value enters G~; G_prev is the rounded G.",
+             "# e.g. bf16(0.3) = 0.30078125, bf16(0.03) = 0.030029296875.",
+             "# columns: step  A11 A22  Gt11 Gt22  M11 M22  Gprev11 Gprev22"]
+    for k, G in enumerate(Gs, 1):
+        Dk = [G[i] - Gp[i] for i in range(2)]
+        A = [bf16(beta * A[i] + (1 - beta) * Dk[i]) for i in range(2)]
+        Gt = [G[i] + alpha * A[i] for i in range(2)]
+        M = [mu * M[i] + Gt[i] for i in range(2)]
+        Gp = [bf16(G[i]) for i in range(2)]
+        lines.append(" ".join([str(k)] + [f"{float(v):.16f}" for v in (A + Gt + M + Gp)]))
+    open(os.path.join(HERE, "hand_lite_2x2.txt"), "w").write("\n".join(lines) + "\n")
+
+
 if __name__ == "__main__":
-    write_orbits(); write_2x2(); write_3x2()
+    write_orbits(); write_2x2(); write_3x2(); write_lite_2x2()

@@ -280,6 +280,60 @@ def check_first_step(orc):
     np.testing.assert_allclose(st.M, 0.5 * G, rtol=1e-13)
 
 
-ALL_CHECKS = [check_scalar_orbits, check_quintic_band, check_hand_2x2, check_hand_3x2,
+def check_bf16_rounding(orc):
+    """MONA-Lite storage: round_bf16 against values fixed by the format (8 significant bits, ties to
+    even) and against an independent library conversion (torch's float32 -> bfloat16)."""
+    import torch
+    exact = [(1.0, 1.0), (1.0 + 2.0 ** -8, 1.0),                       # tie -> even (1.0)
+             (1.0078125 + 2.0 ** -8, 1.015625),                        # tie -> even (1.015625)
+             (1.0 + 2.0 ** -8 + 2.0 ** -20, 1.0078125),                # just above the tie
+             (0.3, 0.30078125), (0.03, 0.030029296875), (-0.3, -0.30078125), (3.0, 3.0), (0.0, 0.0),
+             (1e-3, 0.00099945068359375)]
+    for x, want in exact:
+        got = float(orc.round_bf16(np.array([x]))[0])
+        assert got == want, (x, got, want)
+    rng = np.random.default_rng(11)
+    x = (rng.standard_normal(20000) * np.exp(rng.uniform(-20, 20, 20000))).astype(np.float32)
+    lib = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(orc.round_bf16(x), lib)
+
+
+def check_lite_hand_2x2(orc):
+    """MONA-Lite: two steps on diagonal 2x2 matrices against exact rational arithmetic with bfloat16
+    storage of A_k and G_{k-1} (tests/golden/hand_lite_2x2.txt)."""
+    hp = orc.Hyper(lr=0.1, momentum=0.5, accel_beta=0.9, accel_alpha=-5.0, weight_decay=0.1, ns_steps=5, norm_eps=0.0,
+                   state_dtype="bf16")
+    st = orc.OracleState(2, 2)
+    W = np.diag([1.0, -1.0])
+    Gs = [np.diag([0.3, 3.0]), np.diag([0.3, 4.0])]
+    for row, G in zip(_rows("hand_lite_2x2.txt"), Gs):
+        # what the step sees before it stores: recompute G~ from the stored A
+        W, _ = orc.mona_step(W, G, st, hp)
+        A, Gt, M, Gp = row[1:3], row[3:5], row[5:7], row[7:9]
+        assert np.allclose(np.diag(st.A), A, rtol=0, atol=1e-15), (np.diag(st.A), A)
+        assert np.allclose(np.diag(st.M), M, rtol=0, atol=1e-15), (np.diag(st.M), M)
+        assert np.allclose(np.diag(st.G_prev), Gp, rtol=0, atol=1e-15), (np.diag(st.G_prev), Gp)
+        assert st.A[0, 1] == 0 and st.M[1, 0] == 0
+    # full-precision storage is untouched by the switch: the fp32-state run differs from the Lite run
+    st32 = orc.OracleState(2, 2)
+    hp32 = orc.Hyper(lr=0.1, momentum=0.5, accel_beta=0.9, accel_alpha=-5.0, weight_decay=0.1, ns_steps=5, norm_eps=0.0)
+    orc.mona_step(np.diag([1.0, -1.0]), Gs[0], st32, hp32)
+    assert abs(st32.A[0, 0] - 0.03) < 1e-17 and st32.G_prev[0, 0] == 0.3
+
+
+def check_lite_exactly_representable(orc):
+    """MONA-Lite: when every stored quantity is exactly representable in bfloat16 the Lite trajectory
+    equals the full-precision one (beta_a = 0.5, dyadic gradients)."""
+    g = np.array([[0.5, -0.25], [1.0, 2.0], [0.125, 4.0]])
+    kw = dict(lr=0.1, momentum=0.5, accel_beta=0.5, accel_alpha=-1.0, weight_decay=0.0, ns_steps=2)
+    a, b = orc.OracleState(3, 2), orc.OracleState(3, 2)
+    Wa = Wb = np.ones((3, 2))
+    for k in range(3):
+        Wa, _ = orc.mona_step(Wa, g * (k + 1), a, orc.Hyper(**kw))
+        Wb, _ = orc.mona_step(Wb, g * (k + 1), b, orc.Hyper(state_dtype="bf16", **kw))
+    assert np.array_equal(a.A, b.A) and np.array_equal(a.M, b.M) and np.array_equal(a.G_prev, b.G_prev) and np.array_equal(Wa, Wb)
+
+
+ALL_CHECKS = [check_bf16_rounding, check_lite_hand_2x2, check_lite_exactly_representable, check_scalar_orbits, check_quintic_band, check_hand_2x2, check_hand_3x2,
               check_constant_gradient, check_alpha_zero_is_muon, check_general_step_unrolled,
               check_svd_route_and_brute_force, check_symmetries, check_lemma_bounds, check_first_step]

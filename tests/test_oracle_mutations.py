@@ -28,7 +28,13 @@ MUTATIONS = {
     "decay_outside_lr": ("W - lr * (gamma * O + weight_decay * W)", "W - lr * gamma * O - weight_decay * W"),
     "update_sign": ("W - lr * (gamma * O + weight_decay * W)", "W + lr * (gamma * O + weight_decay * W)"),
     "decay_sign": ("gamma * O + weight_decay * W", "gamma * O - weight_decay * W"),
-    "prev_grad_not_stored": ("state.G_prev = G.copy()", "pass"),
+    "prev_grad_not_stored": ("state.G_prev = store(G.copy())", "pass"),
+    "lite_accel_uses_unrounded_A": ("    A = store(beta_a * A_prev + (1.0 - beta_a) * D)\n    G_tilde = G + alpha * A\n    return A, G_tilde",
+                                    "    A = beta_a * A_prev + (1.0 - beta_a) * D\n    G_tilde = G + alpha * A\n    return store(A), G_tilde"),
+    "lite_prev_grad_not_rounded": ("state.G_prev = store(G.copy())", "state.G_prev = G.copy()"),
+    "lite_momentum_rounded_too": ("    state.M = M\n", "    state.M = store(M)\n"),
+    "lite_round_truncates": ("u = u + 0x7FFF + ((u >> 16) & 1)", "u = u + 0"),
+    "lite_round_half_up": ("u = u + 0x7FFF + ((u >> 16) & 1)", "u = u + 0x8000"),
     "state_M_not_stored": ("state.M = M\n", "pass\n"),
     "coefficient_a": ("NS_A = 3.4445", "NS_A = 3.4454"),
     "coefficient_c": ("NS_C = 2.0315", "NS_C = 2.0351"),
