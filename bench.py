@@ -202,6 +202,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--chunk-mb", type=int, default=None, help="override the chunk budget (MiB)")
     ap.add_argument("--no-overlap", action="store_true", help="keep all chunks on one stream")
+    ap.add_argument("--lite", action="store_true", help="MONA-Lite storage: A_k and G_{k-1} kept in bfloat16")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -229,11 +230,13 @@ def main():
     # every rank owns an independent parameter set of this shape (weak scaling, no data-path collective)
     params = synth.init_params(wl, dev, seed_offset=rank)
     gp = synth.GradientProcess(wl, dev, keep_fp32_shadow=False)
-    opt = pkg.MonaOptimizer(params, grad_dtype=wl.grad_dtype, device=local_rank)
+    opt = pkg.MonaOptimizer(params, grad_dtype=wl.grad_dtype, device=local_rank,
+                            state_dtype=torch.bfloat16 if args.lite else torch.float32)
     hp = pkg.default_hparams(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
     g_elem = 2 if wl.grad_dtype == torch.bfloat16 else 4
+    aux = 2 if args.lite else 4                     # bytes per element of A_k and of G_{k-1}
 
     def barrier():
         torch.cuda.synchronize(dev)
@@ -290,7 +293,8 @@ def main():
 
     peaks, peak_src = load_peaks()
     n = wl.n_params
-    pro_bytes = n * (12 + g_elem + 12 + 2)          # read G, G_prev, A, M; write G_prev, A, M, bf16 X
+    pro_elem = g_elem + 2 * aux + 4 + 2 * aux + 4 + 2   # read G, G_prev, A, M; write G_prev, A, M, bf16 X
+    pro_bytes = n * pro_elem
     upd_bytes = n * (4 + 2 + 4)                     # read W, bf16 O; write W
     pro_gbs = pro_bytes / (ms_pro * 1e-3) / 1e9
     upd_gbs = upd_bytes / (ms_upd * 1e-3) / 1e9
@@ -305,7 +309,7 @@ def main():
                 "traffic_unit": "DRAM bytes per launch (ncu, 93-matrix 768x2048 chunk)",
                 "dense_equivalent_tflops": flops_dense / (ms_ns * 1e-3) / 1e12}
     phases = {"prologue_ms": ms_pro, "prologue_gbs": pro_gbs, "prologue_frac_of_hbm_peak": pro_gbs / peaks["hbm_gbs"],
-              "prologue_frac_of_nominal_8000": pro_gbs / 8000.0, "prologue_bytes_per_elem": 12 + g_elem + 14,
+              "prologue_frac_of_nominal_8000": pro_gbs / 8000.0, "prologue_bytes_per_elem": pro_elem,
               "ns_ms": ms_ns, "ns_tflops_executed": ns_tflops, "update_ms": ms_upd, "update_gbs": upd_gbs,
               "update_frac_of_hbm_peak": upd_gbs / peaks["hbm_gbs"], "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peak_src}
 
@@ -351,7 +355,8 @@ def main():
                 "config": {"workload": wl.name, "config_index": args.config, "matrices": wl.n_matrices, "params": wl.n_params,
                            "grad_dtype": str(wl.grad_dtype).replace("torch.", ""), "gradient_process":
                            f"AR(1) rho={wl.rho} sigma={wl.sigma} {wl.dist}", "ns_steps": hp.ns_steps,
-                           "accel_beta": wl.accel_beta, "accel_alpha": wl.accel_alpha, "parallelism":
+                           "accel_beta": wl.accel_beta, "accel_alpha": wl.accel_alpha,
+                           "state_storage": "bf16 A_k and G_{k-1} (MONA-Lite)" if args.lite else "fp32", "parallelism":
                            "independent parameter set per GPU, no collective" if world > 1 else "single GPU",
                            "l2": "inputs larger than L2 and a 256 MiB buffer rewritten between timed steps",
                            "timing": "CUDA events around each mona_step; gradient refresh between steps untimed",

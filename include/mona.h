@@ -61,7 +61,12 @@ typedef struct {
     int64_t batch;             /* >= 1                                                                */
     int64_t batch_stride;      /* elements between consecutive matrices, >= rows*cols (0 = rows*cols) */
     int32_t grad_dtype;        /* mona_dtype of the gradient                                          */
-    int32_t reserved;
+    int32_t state_dtype;       /* mona_dtype in which A_k and G_{k-1} are stored: MONA_F32 (0, Algorithm 1 as
+                                  printed, "full precision"), or MONA_BF16 = MONA-Lite (section "Efficient
+                                  Deployment with Reduced Overhead"): both buffers kept in bfloat16, equations
+                                  unchanged.  A_k is formed in fp32, rounded to nearest-even once when stored,
+                                  and the stored value is the one G~_k uses; G_{k-1} is the rounded G_k.
+                                  M_k is fp32 either way.                                              */
 } mona_matrix_desc;
 
 /* REQUIRE line of Algorithm 1.  Doubles on purpose: (1 - beta_a), eta*gamma and eta*lambda are formed
@@ -101,8 +106,8 @@ mona_status mona_set_chunk_budget(size_t bytes);
  * every launch on the caller's stream.  Results are identical either way; the workspace holds two chunks. */
 mona_status mona_set_chunk_overlap(int enabled);
 
-/* Bytes the caller must provide for the optimizer state (M, A, G_prev: 3 fp32 per parameter,
- * Algorithm 1 line 1) and for the Newton-Schulz workspace.  Host only; no device is touched. */
+/* Bytes the caller must provide for the optimizer state (M, A, G_prev, Algorithm 1 line 1: 12 bytes per
+ * parameter, 8 with bfloat16 storage of A and G_prev) and for the Newton-Schulz workspace.  Host only; no device is touched. */
 mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc,
                              size_t* state_bytes, size_t* workspace_bytes);
 
@@ -146,8 +151,9 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp,
 mona_status mona_poll_status(mona_handle* h, void* stream, int64_t* first_bad_matrix);
 
 /* Byte offsets inside the state block of M, A and G_prev of matrix 0 of descriptor `desc`.  Matrix b
- * of the descriptor follows at b * rows * cols * 4 bytes from each offset (state is stored densely,
- * whatever batch_stride is).  A checkpoint is the state block plus the caller's own step count. */
+ * of the descriptor follows at b * rows * cols * (element size) bytes from each offset: 4 for M, and 4
+ * or 2 for A and G_prev according to the descriptor's state_dtype (state is stored densely, whatever
+ * batch_stride is).  A checkpoint is the state block plus the caller's own step count. */
 mona_status mona_state_layout(const mona_handle* h, int64_t desc,
                               size_t* off_M, size_t* off_A, size_t* off_Gprev);
 

@@ -24,7 +24,7 @@ class MonaError(RuntimeError):
 
 class MatrixDesc(C.Structure):
     _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("batch", C.c_int64), ("batch_stride", C.c_int64),
-                ("grad_dtype", C.c_int32), ("reserved", C.c_int32)]
+                ("grad_dtype", C.c_int32), ("state_dtype", C.c_int32)]
 
 
 class Hparams(C.Structure):
@@ -124,7 +124,8 @@ class MonaOptimizer:
     `grads[i]` has the same shape in fp32 or bf16.  step() enqueues one optimizer step on the current
     torch stream."""
 
-    def __init__(self, params: Sequence[torch.Tensor], grad_dtype=torch.float32, device: Optional[int] = None):
+    def __init__(self, params: Sequence[torch.Tensor], grad_dtype=torch.float32, device: Optional[int] = None,
+                 state_dtype=torch.float32):
         L = lib()
         self.descs: List[MatrixDesc] = []
         for p in params:
@@ -132,7 +133,8 @@ class MonaOptimizer:
                 raise ValueError("parameters must be contiguous fp32 tensors of shape (rows, cols) or (batch, rows, cols)")
             batch = p.shape[0] if p.dim() == 3 else 1
             rows, cols = p.shape[-2], p.shape[-1]
-            self.descs.append(MatrixDesc(rows, cols, batch, rows * cols, MONA_BF16 if grad_dtype == torch.bfloat16 else MONA_F32, 0))
+            self.descs.append(MatrixDesc(rows, cols, batch, rows * cols, MONA_BF16 if grad_dtype == torch.bfloat16 else MONA_F32,
+                                         MONA_BF16 if state_dtype == torch.bfloat16 else MONA_F32))
         self.device = torch.cuda.current_device() if device is None else device
         self.grad_dtype = grad_dtype
         sb, wb = query_sizes(self.descs)
@@ -181,11 +183,17 @@ class MonaOptimizer:
         return a.value, b.value, c.value
 
     def state_views(self, desc: int):
-        """fp32 views (batch, rows, cols) of M, A, G_prev of descriptor `desc` inside the state block."""
+        """Views (batch, rows, cols) of M, A, G_prev of descriptor `desc` inside the state block: M fp32,
+        A and G_prev in the descriptor's state dtype."""
         d = self.descs[desc]
         n = d.batch * d.rows * d.cols
-        flat = self.state.view(torch.float32)
-        return tuple(flat[off // 4: off // 4 + n].view(d.batch, d.rows, d.cols) for off in self.state_layout(desc))
+        aux = torch.bfloat16 if d.state_dtype == MONA_BF16 else torch.float32
+        offs = self.state_layout(desc)
+        out = []
+        for off, dt in zip(offs, (torch.float32, aux, aux)):
+            sz = 2 if dt == torch.bfloat16 else 4
+            out.append(self.state[off: off + n * sz].view(dt).view(d.batch, d.rows, d.cols))
+        return tuple(out)
 
     def last_launch_count(self) -> int:
         return lib().mona_last_launch_count(self._h)

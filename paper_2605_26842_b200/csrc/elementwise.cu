@@ -37,12 +37,37 @@ struct GradLoad<__nv_bfloat16> {
     static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 };
 
+// Storage format of the two auxiliary buffers A_k and G_{k-1}: fp32, or bfloat16 (MONA-Lite: the value is
+// rounded once, to nearest even, when it is stored, and the stored value is what the step goes on with).
+template <typename ST>
+struct StateIO;
+template <>
+struct StateIO<float> {
+    static __device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ void store4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+    static __device__ __forceinline__ float load1(const float* p) { return *p; }
+    static __device__ __forceinline__ void store1(float* p, float v) { *p = v; }
+    static __device__ __forceinline__ float round(float v) { return v; }
+};
+template <>
+struct StateIO<__nv_bfloat16> {
+    static __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) { return GradLoad<__nv_bfloat16>::load4(p); }
+    static __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {     // v holds already-rounded values
+        __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        __stcs(reinterpret_cast<uint2*>(p), make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi)));
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+    static __device__ __forceinline__ float round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+};
+
+template <typename ST>
 __device__ __forceinline__ void mona_elem(float g, float& gp, float& a, float& m, const PrologueScalars& k) {
     float d = g - gp;                                              // D_k = G_k - G_{k-1}
-    a = mul_add2(k.beta, a, fmaf(k.one_minus_beta.hi, d, k.one_minus_beta.lo * d));  // A_k
+    a = StateIO<ST>::round(mul_add2(k.beta, a, fmaf(k.one_minus_beta.hi, d, k.one_minus_beta.lo * d)));  // A_k as stored
     float gt = mul_add2(k.alpha, a, g);                             // G~_k = G_k + alpha A_k
     m = mul_add2(k.mu, m, gt);                                      // M_k = mu M_{k-1} + G~_k
-    gp = g;                                                         // G_{k-1} <- G_k
+    gp = StateIO<ST>::round(g);                                     // G_{k-1} <- G_k
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -68,9 +93,9 @@ __device__ __forceinline__ float block_sum(float v, float* smem /* >= 8 floats *
 // grid = (slabs, C).  Block (p, c) owns elements [p*slab_len, min(e, (p+1)*slab_len)) of matrix c.
 // The last block of a matrix to finish adds the slab partials in index order, so ||M||_F does not
 // depend on scheduling; it then resets the arrival counter for the next call.
-template <typename GT, int VEC>
+template <typename GT, typename ST, int VEC>
 __global__ void __launch_bounds__(EW_THREADS)
-prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, float* __restrict__ Ast, float* __restrict__ Gpst,
+prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, ST* __restrict__ Gpst,
                 __nv_bfloat16* __restrict__ xhat, float* __restrict__ partials, unsigned int* __restrict__ counters,
                 float* __restrict__ inv_norm, DeviceStatus* __restrict__ status, long long e, long long slab_len,
                 int slabs, PrologueScalars k) {
@@ -81,8 +106,8 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, float* __restrict__ Ast
     const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
     const GT* __restrict__ g = reinterpret_cast<const GT*>(ptrs.g[c]);
     float* __restrict__ M = Mst + (long long)c * e;
-    float* __restrict__ A = Ast + (long long)c * e;
-    float* __restrict__ Gp = Gpst + (long long)c * e;
+    ST* __restrict__ A = Ast + (long long)c * e;
+    ST* __restrict__ Gp = Gpst + (long long)c * e;
     __nv_bfloat16* __restrict__ X = xhat ? xhat + (long long)c * e : nullptr;
 
     float acc = 0.f;
@@ -92,15 +117,15 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, float* __restrict__ Ast
         // two independent vectors per trip keep ~128 B per thread in flight
         for (; i + STEP < hi; i += 2 * STEP) {
             float4 g0 = GradLoad<GT>::load4(g + i), g1 = GradLoad<GT>::load4(g + i + STEP);
-            float4 p0 = __ldcs(reinterpret_cast<const float4*>(Gp + i)), p1 = __ldcs(reinterpret_cast<const float4*>(Gp + i + STEP));
-            float4 a0 = __ldcs(reinterpret_cast<const float4*>(A + i)), a1 = __ldcs(reinterpret_cast<const float4*>(A + i + STEP));
+            float4 p0 = StateIO<ST>::load4(Gp + i), p1 = StateIO<ST>::load4(Gp + i + STEP);
+            float4 a0 = StateIO<ST>::load4(A + i), a1 = StateIO<ST>::load4(A + i + STEP);
             float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i)), m1 = __ldcs(reinterpret_cast<const float4*>(M + i + STEP));
-            mona_elem(g0.x, p0.x, a0.x, m0.x, k); mona_elem(g0.y, p0.y, a0.y, m0.y, k);
-            mona_elem(g0.z, p0.z, a0.z, m0.z, k); mona_elem(g0.w, p0.w, a0.w, m0.w, k);
-            mona_elem(g1.x, p1.x, a1.x, m1.x, k); mona_elem(g1.y, p1.y, a1.y, m1.y, k);
-            mona_elem(g1.z, p1.z, a1.z, m1.z, k); mona_elem(g1.w, p1.w, a1.w, m1.w, k);
-            __stcs(reinterpret_cast<float4*>(Gp + i), p0); __stcs(reinterpret_cast<float4*>(Gp + i + STEP), p1);
-            __stcs(reinterpret_cast<float4*>(A + i), a0);  __stcs(reinterpret_cast<float4*>(A + i + STEP), a1);
+            mona_elem<ST>(g0.x, p0.x, a0.x, m0.x, k); mona_elem<ST>(g0.y, p0.y, a0.y, m0.y, k);
+            mona_elem<ST>(g0.z, p0.z, a0.z, m0.z, k); mona_elem<ST>(g0.w, p0.w, a0.w, m0.w, k);
+            mona_elem<ST>(g1.x, p1.x, a1.x, m1.x, k); mona_elem<ST>(g1.y, p1.y, a1.y, m1.y, k);
+            mona_elem<ST>(g1.z, p1.z, a1.z, m1.z, k); mona_elem<ST>(g1.w, p1.w, a1.w, m1.w, k);
+            StateIO<ST>::store4(Gp + i, p0); StateIO<ST>::store4(Gp + i + STEP, p1);
+            StateIO<ST>::store4(A + i, a0);  StateIO<ST>::store4(A + i + STEP, a1);
             __stcs(reinterpret_cast<float4*>(M + i), m0);  __stcs(reinterpret_cast<float4*>(M + i + STEP), m1);
             if (X) {
                 *reinterpret_cast<uint2*>(X + i) = make_uint2(pack_bf16x2(m0.x, m0.y), pack_bf16x2(m0.z, m0.w));
@@ -111,22 +136,22 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, float* __restrict__ Ast
         }
         for (; i < hi; i += STEP) {
             float4 g0 = GradLoad<GT>::load4(g + i);
-            float4 p0 = __ldcs(reinterpret_cast<const float4*>(Gp + i));
-            float4 a0 = __ldcs(reinterpret_cast<const float4*>(A + i));
+            float4 p0 = StateIO<ST>::load4(Gp + i);
+            float4 a0 = StateIO<ST>::load4(A + i);
             float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i));
-            mona_elem(g0.x, p0.x, a0.x, m0.x, k); mona_elem(g0.y, p0.y, a0.y, m0.y, k);
-            mona_elem(g0.z, p0.z, a0.z, m0.z, k); mona_elem(g0.w, p0.w, a0.w, m0.w, k);
-            __stcs(reinterpret_cast<float4*>(Gp + i), p0);
-            __stcs(reinterpret_cast<float4*>(A + i), a0);
+            mona_elem<ST>(g0.x, p0.x, a0.x, m0.x, k); mona_elem<ST>(g0.y, p0.y, a0.y, m0.y, k);
+            mona_elem<ST>(g0.z, p0.z, a0.z, m0.z, k); mona_elem<ST>(g0.w, p0.w, a0.w, m0.w, k);
+            StateIO<ST>::store4(Gp + i, p0);
+            StateIO<ST>::store4(A + i, a0);
             __stcs(reinterpret_cast<float4*>(M + i), m0);
             if (X) *reinterpret_cast<uint2*>(X + i) = make_uint2(pack_bf16x2(m0.x, m0.y), pack_bf16x2(m0.z, m0.w));
             acc = fmaf(m0.x, m0.x, acc); acc = fmaf(m0.y, m0.y, acc); acc = fmaf(m0.z, m0.z, acc); acc = fmaf(m0.w, m0.w, acc);
         }
     } else {
         for (long long i = lo + threadIdx.x; i < hi; i += EW_THREADS) {
-            float gv = GradLoad<GT>::load1(g + i), pv = Gp[i], av = A[i], mv = M[i];
-            mona_elem(gv, pv, av, mv, k);
-            Gp[i] = pv; A[i] = av; M[i] = mv;
+            float gv = GradLoad<GT>::load1(g + i), pv = StateIO<ST>::load1(Gp + i), av = StateIO<ST>::load1(A + i), mv = M[i];
+            mona_elem<ST>(gv, pv, av, mv, k);
+            StateIO<ST>::store1(Gp + i, pv); StateIO<ST>::store1(A + i, av); M[i] = mv;
             if (X) X[i] = __float2bfloat16_rn(mv);
             acc = fmaf(mv, mv, acc);
         }
@@ -202,17 +227,27 @@ scale_kernel(const float* __restrict__ M, float* __restrict__ X, const float* __
 
 }  // namespace
 
-cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool vec4, float* M, float* A, float* Gp,
+namespace {
+template <typename GT, typename ST>
+void launch_prologue_t(dim3 grid, dim3 block, cudaStream_t stream, bool vec4, const ChunkPtrs& ptrs, float* M, void* A, void* Gp,
+                       __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm, DeviceStatus* status,
+                       long long e, long long slab_len, int slabs, const PrologueScalars& k) {
+    if (vec4) prologue_kernel<GT, ST, 4><<<grid, block, 0, stream>>>(ptrs, M, (ST*)A, (ST*)Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+    else      prologue_kernel<GT, ST, 1><<<grid, block, 0, stream>>>(ptrs, M, (ST*)A, (ST*)Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+}
+}  // namespace
+
+cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool state_bf16, bool vec4, float* M, void* A, void* Gp,
                             __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm,
                             DeviceStatus* status, long long e, long long slab_len, int slabs,
                             const PrologueScalars& k, cudaStream_t stream) {
     dim3 grid(slabs, C), block(EW_THREADS);
     if (grad_bf16) {
-        if (vec4) prologue_kernel<__nv_bfloat16, 4><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
-        else      prologue_kernel<__nv_bfloat16, 1><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        if (state_bf16) launch_prologue_t<__nv_bfloat16, __nv_bfloat16>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        else            launch_prologue_t<__nv_bfloat16, float>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
     } else {
-        if (vec4) prologue_kernel<float, 4><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
-        else      prologue_kernel<float, 1><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        if (state_bf16) launch_prologue_t<float, __nv_bfloat16>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        else            launch_prologue_t<float, float>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
     }
     return cudaGetLastError();
 }
@@ -337,7 +372,7 @@ extern "C" mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtyp
     k.alpha = split_double(hp->accel_alpha);
     k.mu = split_double(hp->momentum);
     k.eps = (float)hp->norm_eps;
-    ce = launch_prologue(ptrs, 1, grad_dtype == MONA_BF16, e % 4 == 0, M, A, G_prev, (__nv_bfloat16*)xhat_bf16, scratch->partials,
+    ce = launch_prologue(ptrs, 1, grad_dtype == MONA_BF16, false, e % 4 == 0, M, A, G_prev, (__nv_bfloat16*)xhat_bf16, scratch->partials,
                          &scratch->counter, inv_norm_out, &scratch->status, e, slab, slabs, k, stream);
     if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
     set_msg(err, err_len, "");

@@ -6,9 +6,10 @@ namespace mona {
 
 // Fused prologue over a chunk of C same-shape matrices (state stored densely, e elements each):
 // updates A, M, G_prev in place from the gradient, optionally writes bf16(M) to `xhat` (null to skip),
-// and leaves 1/(||M||_F + eps) of matrix c in inv_norm[c].  `partials` holds C*MAX_SLABS floats and
+// and leaves 1/(||M||_F + eps) of matrix c in inv_norm[c].  A and G_prev are fp32, or bfloat16 when
+// `state_bf16` (MONA-Lite storage); M is always fp32.  `partials` holds C*MAX_SLABS floats and
 // `counters` C zero-initialised words of scratch.
-cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool vec4, float* M, float* A, float* Gp,
+cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool state_bf16, bool vec4, float* M, void* A, void* Gp,
                             __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm,
                             DeviceStatus* status, long long e, long long slab_len, int slabs,
                             const PrologueScalars& k, cudaStream_t stream);

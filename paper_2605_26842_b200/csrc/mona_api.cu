@@ -57,10 +57,11 @@ struct MatRef {
 
 struct Bucket {
     int64_t rows = 0, cols = 0, s = 0, l = 0, e = 0;
-    int grad_dtype = 0;
+    int grad_dtype = 0, state_dtype = 0;
     bool tall = false, tc_ok = false;
     std::vector<MatRef> mats;
-    int64_t state_off = 0;      // floats from the state base: M block, then A block, then G_prev block
+    // bytes from the state base of the three blocks: M (fp32), A and G_prev (fp32, or bf16 with MONA-Lite storage)
+    size_t off_M = 0, off_A = 0, off_G = 0;
     int Cb = 1, Cf = 1;         // chunk capacity: bf16 tensor-core mode / fp32 mode
     int slabs = 1;
     int64_t slab_len = 0;
@@ -82,23 +83,24 @@ struct Plan {
 mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan, std::string& err) {
     if (!descs || n_desc <= 0) { err = "descs is null or n_desc <= 0"; return MONA_ERR_INVALID_ARG; }
     plan.descs.assign(descs, descs + n_desc);
-    std::map<std::tuple<int64_t, int64_t, int>, int> index;
+    std::map<std::tuple<int64_t, int64_t, int, int>, int> index;
     int64_t gid = 0;
     for (int64_t i = 0; i < n_desc; ++i) {
         mona_matrix_desc& d = plan.descs[i];
         if (d.rows <= 0 || d.cols <= 0 || d.batch <= 0) { err = "descriptor with non-positive rows/cols/batch"; return MONA_ERR_INVALID_ARG; }
         if (d.grad_dtype != MONA_F32 && d.grad_dtype != MONA_BF16) { err = "descriptor with unknown grad_dtype"; return MONA_ERR_INVALID_ARG; }
+        if (d.state_dtype != MONA_F32 && d.state_dtype != MONA_BF16) { err = "descriptor with unknown state_dtype"; return MONA_ERR_INVALID_ARG; }
         if (d.rows > (1 << 20) || d.cols > (1 << 20) || d.rows * d.cols > (1ll << 31)) { err = "matrix too large"; return MONA_ERR_UNSUPPORTED_SHAPE; }
         if (d.batch_stride == 0) d.batch_stride = d.rows * d.cols;
         if (d.batch_stride < d.rows * d.cols) { err = "batch_stride smaller than rows*cols"; return MONA_ERR_INVALID_ARG; }
-        auto key = std::make_tuple(d.rows, d.cols, (int)d.grad_dtype);
+        auto key = std::make_tuple(d.rows, d.cols, (int)d.grad_dtype, (int)d.state_dtype);
         auto it = index.find(key);
         int bi;
         if (it == index.end()) {
             bi = (int)plan.buckets.size();
             index[key] = bi;
             Bucket b;
-            b.rows = d.rows; b.cols = d.cols; b.grad_dtype = d.grad_dtype;
+            b.rows = d.rows; b.cols = d.cols; b.grad_dtype = d.grad_dtype; b.state_dtype = d.state_dtype;
             b.tall = d.rows > d.cols;
             b.s = std::min(d.rows, d.cols); b.l = std::max(d.rows, d.cols); b.e = d.rows * d.cols;
             // below 64 rows bf16 iterates of very wide matrices drift past the 2e-2 bound (measured 2.0-2.4e-2 at 32 x 1024),
@@ -114,13 +116,14 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         for (int64_t b = 0; b < d.batch; ++b) plan.buckets[bi].mats.push_back({(int)i, b});
         gid += d.batch;
     }
-    int64_t state_floats = 0;
+    size_t state_bytes = 0;
     size_t max_data = 0;
     for (Bucket& b : plan.buckets) {
         const int64_t count = (int64_t)b.mats.size();
-        b.state_off = state_floats;
-        state_floats += 3 * count * b.e;
-        state_floats = (int64_t)align_up((size_t)state_floats, 64);        // keep every block 256-byte aligned
+        const size_t aux = b.state_dtype == MONA_BF16 ? 2 : 4;              // every block starts 256-byte aligned
+        b.off_M = state_bytes; state_bytes += align_up((size_t)count * b.e * 4, 256);
+        b.off_A = state_bytes; state_bytes += align_up((size_t)count * b.e * aux, 256);
+        b.off_G = state_bytes; state_bytes += align_up((size_t)count * b.e * aux, 256);
         // slabs: ~16K elements each, at most MAX_SLABS, slab length a multiple of 1024
         int64_t slab = 16384;
         if ((b.e + slab - 1) / slab > MAX_SLABS) slab = (int64_t)align_up((size_t)((b.e + MAX_SLABS - 1) / MAX_SLABS), 1024);
@@ -143,7 +146,7 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         b.data_bytes = std::max(off, off32);
         max_data = std::max(max_data, b.data_bytes);
     }
-    plan.state_bytes = (size_t)state_floats * 4;
+    plan.state_bytes = state_bytes;
     plan.slot_bytes = align_up(max_data, 1024);
     plan.workspace_bytes = WS_DATA_OFF + NSLOTS * plan.slot_bytes;
     return MONA_OK;
@@ -339,10 +342,9 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
         const int64_t count = (int64_t)b.mats.size();
         const double gamma = hp->scale_mode == 0 ? hp->scale_value * std::sqrt((double)b.l) : hp->scale_value;
         const float eta_gamma = (float)(hp->lr * gamma);
-        float* Mst = (float*)h->state + b.state_off;
-        float* Ast = Mst + count * b.e;
-        float* Gst = Ast + count * b.e;
         const size_t gsz = b.grad_dtype == MONA_BF16 ? 2 : 4;
+        const size_t aux = b.state_dtype == MONA_BF16 ? 2 : 4;
+        float* Mst = (float*)(h->state + b.off_M);
 
         for (int64_t start = 0; start < count; start += cap) {
             const int C = (int)std::min<int64_t>(cap, count - start);
@@ -366,8 +368,8 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             float* inv_norm = (float*)(ctrl + CTRL_INVNORM_OFF);
             float* partials = (float*)(ctrl + CTRL_PARTIALS_OFF);
             float* Mc = Mst + start * b.e;
-            float* Ac = Ast + start * b.e;
-            float* Gc = Gst + start * b.e;
+            void* Ac = h->state + b.off_A + (size_t)start * b.e * aux;
+            void* Gc = h->state + b.off_G + (size_t)start * b.e * aux;
             __nv_bfloat16* xb[2] = {(__nv_bfloat16*)(data + b.off_x[0]), (__nv_bfloat16*)(data + b.off_x[1])};
             __nv_bfloat16* ab = (__nv_bfloat16*)(data + b.off_a);
             float* xf[2] = {(float*)(data + b.off32_x[0]), (float*)(data + b.off32_x[1])};
@@ -375,7 +377,7 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             float* bf = (float*)(data + b.off32_b);
 
             if (phase_mask & 1u) {
-                MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16, vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
+                MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16, b.state_dtype == MONA_BF16, vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
                                              counters, inv_norm, dstatus, b.e, b.slab_len, b.slabs, ps, stream));
                 ++h->launches;
             }
@@ -512,11 +514,11 @@ mona_status mona_poll_status(mona_handle* h, void* stream_v, int64_t* first_bad_
 mona_status mona_state_layout(const mona_handle* h, int64_t desc, size_t* off_M, size_t* off_A, size_t* off_Gprev) {
     if (!h || desc < 0 || desc >= (int64_t)h->plan.descs.size()) return MONA_ERR_INVALID_ARG;
     const Bucket& b = h->plan.buckets[h->plan.desc_bucket[desc]];
-    const int64_t count = (int64_t)b.mats.size();
-    const int64_t base = b.state_off + h->plan.desc_pos[desc] * b.e;
-    if (off_M) *off_M = (size_t)base * 4;
-    if (off_A) *off_A = (size_t)(base + count * b.e) * 4;
-    if (off_Gprev) *off_Gprev = (size_t)(base + 2 * count * b.e) * 4;
+    const size_t aux = b.state_dtype == MONA_BF16 ? 2 : 4;
+    const size_t pos = (size_t)h->plan.desc_pos[desc] * (size_t)b.e;
+    if (off_M) *off_M = b.off_M + pos * 4;
+    if (off_A) *off_A = b.off_A + pos * aux;
+    if (off_Gprev) *off_Gprev = b.off_G + pos * aux;
     return MONA_OK;
 }
 

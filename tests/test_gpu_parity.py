@@ -3,7 +3,8 @@ import pytest
 import torch
 
 import paper_2605_26842_b200 as pkg
-from tests.parity_util import TOL_O_BF16, TOL_O_FP32, TOL_STATE, TOL_W, run_case
+from tests.parity_util import (LITE_MAX_FLIPPED, TOL_A_LITE, TOL_M_LITE, TOL_O_BF16, TOL_O_FP32, TOL_STATE, TOL_W,
+                               run_case)
 
 pytestmark = pytest.mark.gpu
 
@@ -82,6 +83,21 @@ def test_fixed_scale_and_other_hyperparameters():
                              accel_beta=0.9, accel_alpha=-5.0)
     errs = run_case([(1, 256, 256)], steps=3, hp=hp, seed=13)
     check(errs, TOL_O_BF16)
+
+
+@pytest.mark.parametrize("shapes,grad_dtype,steps", [([(1, 256, 512)], torch.float32, 5), ([(2, 512, 256), (1, 32, 1024)], torch.float32, 10),
+                                                     ([(3, 128, 384)], torch.bfloat16, 4), ([(1, 33, 17)], torch.float32, 3)])
+def test_mona_lite_state_storage(shapes, grad_dtype, steps):
+    """MONA-Lite: A_k and G_{k-1} stored in bfloat16.  G_prev must equal the oracle's bit for bit (with
+    bfloat16 gradients it is the gradient itself); A may sit one bfloat16 step away on a small fraction of
+    the elements (the value that is rounded is formed in fp32 here and in fp64 in the oracle), never more."""
+    errs = run_case(shapes, steps=steps, grad_dtype=grad_dtype, seed=21, lite=True)
+    assert errs["Gprev_exact"], errs
+    # a disagreement is made of roundings that went the other way: at most one fresh bfloat16 step per step taken
+    # (measured at the scale of the EMA's operands), on a small fraction of the elements
+    assert errs["A_worst_steps"] <= steps + 1 and errs["A_flipped"] <= LITE_MAX_FLIPPED, errs
+    assert errs["A"] <= TOL_A_LITE and errs["M"] <= TOL_M_LITE, errs
+    assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
 
 
 def test_nonfinite_gradient_is_reported():
