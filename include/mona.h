@@ -84,7 +84,10 @@ typedef struct {
     int32_t scale_mode;    /* 0: gamma = scale_value * sqrt(max(m,n)); 1: gamma = scale_value         */
     int32_t ns_precision;  /* 0: bf16 operands on the tensor cores, fp32 accumulate;
                               1: fp32 validation mode (plain FMA, no tensor cores)                    */
-    int32_t reserved;
+    int32_t algorithm;     /* 0: MONA (Algorithm 1).  1: plain Muon, the baseline of Eq. muon_momentum /
+                              muon_ns / muon_update: M_k = mu M_{k-1} + G_k, same orthogonalisation and
+                              update; accel_beta and accel_alpha are ignored and A, G_prev are neither read
+                              nor written (they keep whatever they held).                             */
 } mona_hparams;
 
 typedef struct mona_handle mona_handle;

@@ -13,6 +13,7 @@ notation, with no blocking, fusion or reordering:
   * Eq. newton_schulz                       -> newton_schulz(): X_0 = M/||M||_F, quintic iteration
   * gamma = 0.2 sqrt(max(m, n))             -> update_scale()
   * Eq. muon_update                         -> apply_update(): W <- W - eta (gamma O + lambda W)
+  * plain Muon, the baseline (Eq. muon_momentum, muon_ns, muon_update)        -> muon_step()
   * MONA-Lite (section "Efficient Deployment with Reduced Overhead"): G_{k-1} and A_k kept in
     bfloat16, equations unchanged          -> round_bf16(), Hyper.state_dtype = "bf16"
 
@@ -143,4 +144,18 @@ def mona_step(W, G, state: OracleState, hp: Hyper):
     state.A = A
     state.M = M
     state.G_prev = store(G.copy())   # Algorithm 1, line 10
+    return W_next, O
+
+
+def muon_step(W, G, state: OracleState, hp: Hyper):
+    """One step of plain Muon for one matrix, the baseline the paper compares with:
+    Eq. muon_momentum M_k = mu M_{k-1} + G_k, Eq. muon_ns O_k = NewtonSchulz(M_k, T), Eq. muon_update.
+    Only state.M is used and updated."""
+    W = np.asarray(W, dtype=np.float64)
+    G = np.asarray(G, dtype=np.float64)
+    M = momentum(state.M, G, hp.momentum)
+    O = newton_schulz(M, hp.ns_steps, hp.ns_a, hp.ns_b, hp.ns_c, hp.norm_eps)
+    gamma = update_scale(W.shape[0], W.shape[1], hp.scale_mode, hp.scale_value)
+    W_next = apply_update(W, O, hp.lr, gamma, hp.weight_decay)
+    state.M = M
     return W_next, O

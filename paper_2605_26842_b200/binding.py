@@ -31,7 +31,7 @@ class Hparams(C.Structure):
     _fields_ = [("lr", C.c_double), ("momentum", C.c_double), ("accel_beta", C.c_double), ("accel_alpha", C.c_double),
                 ("weight_decay", C.c_double), ("ns_a", C.c_double), ("ns_b", C.c_double), ("ns_c", C.c_double),
                 ("norm_eps", C.c_double), ("scale_value", C.c_double), ("ns_steps", C.c_int32), ("scale_mode", C.c_int32),
-                ("ns_precision", C.c_int32), ("reserved", C.c_int32)]
+                ("ns_precision", C.c_int32), ("algorithm", C.c_int32)]
 
 
 _lib = None

@@ -61,13 +61,29 @@ struct StateIO<__nv_bfloat16> {
     static __device__ __forceinline__ float round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 };
 
+// Tag for the plain Muon step (Eq. muon_momentum): there is no acceleration state to read or write.
+struct NoAux {};
+template <>
+struct StateIO<NoAux> {
+    static __device__ __forceinline__ float4 load4(const NoAux*) { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ void store4(NoAux*, float4) {}
+    static __device__ __forceinline__ float load1(const NoAux*) { return 0.f; }
+    static __device__ __forceinline__ void store1(NoAux*, float) {}
+    static __device__ __forceinline__ float round(float v) { return v; }
+};
+
 template <typename ST>
 __device__ __forceinline__ void mona_elem(float g, float& gp, float& a, float& m, const PrologueScalars& k) {
+
     float d = g - gp;                                              // D_k = G_k - G_{k-1}
     a = StateIO<ST>::round(mul_add2(k.beta, a, fmaf(k.one_minus_beta.hi, d, k.one_minus_beta.lo * d)));  // A_k as stored
     float gt = mul_add2(k.alpha, a, g);                             // G~_k = G_k + alpha A_k
     m = mul_add2(k.mu, m, gt);                                      // M_k = mu M_{k-1} + G~_k
     gp = StateIO<ST>::round(g);                                     // G_{k-1} <- G_k
+}
+template <>
+__device__ __forceinline__ void mona_elem<NoAux>(float g, float&, float&, float& m, const PrologueScalars& k) {
+    m = mul_add2(k.mu, m, g);                                       // Eq. muon_momentum: M_k = mu M_{k-1} + G_k
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -106,8 +122,8 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, S
     const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
     const GT* __restrict__ g = reinterpret_cast<const GT*>(ptrs.g[c]);
     float* __restrict__ M = Mst + (long long)c * e;
-    ST* __restrict__ A = Ast + (long long)c * e;
-    ST* __restrict__ Gp = Gpst + (long long)c * e;
+    ST* __restrict__ A = Ast ? Ast + (long long)c * e : nullptr;      // pointer arithmetic only; NoAux never dereferences
+    ST* __restrict__ Gp = Gpst ? Gpst + (long long)c * e : nullptr;
     __nv_bfloat16* __restrict__ X = xhat ? xhat + (long long)c * e : nullptr;
 
     float acc = 0.f;
@@ -237,18 +253,22 @@ void launch_prologue_t(dim3 grid, dim3 block, cudaStream_t stream, bool vec4, co
 }
 }  // namespace
 
-cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, bool state_bf16, bool vec4, float* M, void* A, void* Gp,
+cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, int state_kind, bool vec4, float* M, void* A, void* Gp,
                             __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm,
                             DeviceStatus* status, long long e, long long slab_len, int slabs,
                             const PrologueScalars& k, cudaStream_t stream) {
     dim3 grid(slabs, C), block(EW_THREADS);
+#define MONA_PROLOGUE_CASE(GT, ST) launch_prologue_t<GT, ST>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k)
     if (grad_bf16) {
-        if (state_bf16) launch_prologue_t<__nv_bfloat16, __nv_bfloat16>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
-        else            launch_prologue_t<__nv_bfloat16, float>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        if (state_kind == PROLOGUE_NO_AUX) MONA_PROLOGUE_CASE(__nv_bfloat16, NoAux);
+        else if (state_kind == PROLOGUE_AUX_BF16) MONA_PROLOGUE_CASE(__nv_bfloat16, __nv_bfloat16);
+        else MONA_PROLOGUE_CASE(__nv_bfloat16, float);
     } else {
-        if (state_bf16) launch_prologue_t<float, __nv_bfloat16>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
-        else            launch_prologue_t<float, float>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+        if (state_kind == PROLOGUE_NO_AUX) MONA_PROLOGUE_CASE(float, NoAux);
+        else if (state_kind == PROLOGUE_AUX_BF16) MONA_PROLOGUE_CASE(float, __nv_bfloat16);
+        else MONA_PROLOGUE_CASE(float, float);
     }
+#undef MONA_PROLOGUE_CASE
     return cudaGetLastError();
 }
 
@@ -372,7 +392,7 @@ extern "C" mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtyp
     k.alpha = split_double(hp->accel_alpha);
     k.mu = split_double(hp->momentum);
     k.eps = (float)hp->norm_eps;
-    ce = launch_prologue(ptrs, 1, grad_dtype == MONA_BF16, false, e % 4 == 0, M, A, G_prev, (__nv_bfloat16*)xhat_bf16, scratch->partials,
+    ce = launch_prologue(ptrs, 1, grad_dtype == MONA_BF16, PROLOGUE_AUX_F32, e % 4 == 0, M, A, G_prev, (__nv_bfloat16*)xhat_bf16, scratch->partials,
                          &scratch->counter, inv_norm_out, &scratch->status, e, slab, slabs, k, stream);
     if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
     set_msg(err, err_len, "");

@@ -298,6 +298,7 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
     if (hp->ns_steps < 0 || hp->ns_steps > 64) return h->fail(MONA_ERR_INVALID_ARG, "ns_steps out of range");
     if (hp->ns_precision != 0 && hp->ns_precision != 1) return h->fail(MONA_ERR_INVALID_ARG, "ns_precision must be 0 or 1");
     if (hp->scale_mode != 0 && hp->scale_mode != 1) return h->fail(MONA_ERR_INVALID_ARG, "scale_mode must be 0 or 1");
+    if (hp->algorithm != 0 && hp->algorithm != 1) return h->fail(MONA_ERR_INVALID_ARG, "algorithm must be 0 (MONA) or 1 (Muon)");
     const Plan& plan = h->plan;
     const int64_t n_desc = (int64_t)plan.descs.size();
     for (int64_t i = 0; i < n_desc; ++i) {
@@ -377,7 +378,8 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             float* bf = (float*)(data + b.off32_b);
 
             if (phase_mask & 1u) {
-                MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16, b.state_dtype == MONA_BF16, vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
+                MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16,
+                                             hp->algorithm == 1 ? PROLOGUE_NO_AUX : (b.state_dtype == MONA_BF16 ? PROLOGUE_AUX_BF16 : PROLOGUE_AUX_F32), vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
                                              counters, inv_norm, dstatus, b.e, b.slab_len, b.slabs, ps, stream));
                 ++h->launches;
             }

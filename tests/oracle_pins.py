@@ -334,6 +334,24 @@ def check_lite_exactly_representable(orc):
     assert np.array_equal(a.A, b.A) and np.array_equal(a.M, b.M) and np.array_equal(a.G_prev, b.G_prev) and np.array_equal(Wa, Wb)
 
 
-ALL_CHECKS = [check_bf16_rounding, check_lite_hand_2x2, check_lite_exactly_representable, check_scalar_orbits, check_quintic_band, check_hand_2x2, check_hand_3x2,
+def check_muon_step(orc):
+    """Plain Muon (Eq. muon_momentum / muon_ns / muon_update): three steps against the separately written
+    reference above, whose orthogonalisation goes through the SVD closed form; A and G_prev stay untouched."""
+    rng = np.random.default_rng(3)
+    hp = orc.Hyper(lr=0.02, momentum=0.9, weight_decay=0.05, norm_eps=0.0)
+    for (m, n) in [(4, 7), (6, 3)]:
+        W = rng.standard_normal((m, n)) * 0.1
+        Wr, Mr = W.copy(), np.zeros((m, n))
+        st = orc.OracleState(m, n)
+        for _ in range(3):
+            G = rng.standard_normal((m, n))
+            W, O = orc.muon_step(W, G, st, hp)
+            Wr, Mr, Or = muon_reference_step(Wr, G, Mr, hp.lr, hp.momentum, hp.weight_decay, 0.2 * np.sqrt(max(m, n)))
+            assert np.allclose(st.M, Mr, rtol=0, atol=1e-13) and np.allclose(O, Or, rtol=0, atol=1e-10)
+            assert np.allclose(W, Wr, rtol=0, atol=1e-12)
+        assert not st.A.any() and not st.G_prev.any()
+
+
+ALL_CHECKS = [check_muon_step, check_bf16_rounding, check_lite_hand_2x2, check_lite_exactly_representable, check_scalar_orbits, check_quintic_band, check_hand_2x2, check_hand_3x2,
               check_constant_gradient, check_alpha_zero_is_muon, check_general_step_unrolled,
               check_svd_route_and_brute_force, check_symmetries, check_lemma_bounds, check_first_step]

@@ -59,7 +59,7 @@ def ar1_grads(shapes, steps, rho, sigma, seed, dtype=torch.float32, heavy_tail=F
 
 
 def run_case(shapes, steps=3, hp=None, grad_dtype=torch.float32, rho=0.9, sigma=1e-3, seed=0, heavy_tail=False,
-             pad=0, sample=None, lite=False):
+             pad=0, sample=None, lite=False, muon=False):
     """shapes: list of (batch, rows, cols).  `pad` adds that many elements between stacked matrices
     (batch_stride > rows*cols).  `sample`: dict spec index -> list of batch indices the oracle follows
     (default: all).  Returns dict of max relative errors over steps and sampled matrices."""
@@ -103,7 +103,8 @@ def run_case(shapes, steps=3, hp=None, grad_dtype=torch.float32, rho=0.9, sigma=
             Mv, Av, Gv = opt.state_views(i)
             for b in sample[i]:
                 A_before[(i, b)] = states[(i, b)].A.copy()
-                Wn, O = orc.mona_step(Wref[(i, b)], grads_seq[k][i][b].double().numpy(), states[(i, b)], ohp)
+                step_fn = orc.muon_step if muon else orc.mona_step
+                Wn, O = step_fn(Wref[(i, b)], grads_seq[k][i][b].double().numpy(), states[(i, b)], ohp)
                 Wref[(i, b)] = Wn
                 s = states[(i, b)]
                 a_gpu, g_gpu = Av[b].double().cpu().numpy(), Gv[b].double().cpu().numpy()

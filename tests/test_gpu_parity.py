@@ -100,6 +100,15 @@ def test_mona_lite_state_storage(shapes, grad_dtype, steps):
     assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
 
 
+def test_plain_muon_path():
+    """algorithm = 1: Eq. muon_momentum without the acceleration term; A and G_prev are neither read nor written
+    (they stay at their initial zero, so their error against the oracle's untouched zero state is exactly 0)."""
+    hp = pkg.default_hparams(algorithm=1)
+    errs = run_case([(2, 256, 384), (1, 384, 128), (1, 40, 72)], steps=4, hp=hp, seed=17, muon=True)
+    assert errs["A"] == 0.0 and errs["Gprev"] == 0.0, errs
+    check(errs, TOL_O_BF16)
+
+
 def test_nonfinite_gradient_is_reported():
     dev = torch.device("cuda", 0)
     p = [torch.zeros(2, 128, 128, device=dev), torch.zeros(1, 64, 64, device=dev)]

@@ -34,6 +34,8 @@ MUTATIONS = {
     "lite_prev_grad_not_rounded": ("state.G_prev = store(G.copy())", "state.G_prev = G.copy()"),
     "lite_momentum_rounded_too": ("    state.M = M\n", "    state.M = store(M)\n"),
     "lite_round_truncates": ("u = u + 0x7FFF + ((u >> 16) & 1)", "u = u + 0"),
+    "muon_step_forgets_momentum": ("    state.M = M\n    return W_next, O\n", "    return W_next, O\n"),
+    "muon_step_adds_acceleration": ("    M = momentum(state.M, G, hp.momentum)\n    O = newton_schulz(M, hp.ns_steps", "    M = momentum(state.M, G + hp.accel_alpha * (1.0 - hp.accel_beta) * G, hp.momentum)\n    O = newton_schulz(M, hp.ns_steps"),
     "lite_round_half_up": ("u = u + 0x7FFF + ((u >> 16) & 1)", "u = u + 0x8000"),
     "state_M_not_stored": ("state.M = M\n", "pass\n"),
     "coefficient_a": ("NS_A = 3.4445", "NS_A = 3.4454"),
