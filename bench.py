@@ -155,8 +155,8 @@ def pick_workload(index, layers, free_bytes):
     from paper_2605_26842_b200 import synth
     wl = synth.workload(index, layers)
     note = ""
-    if layers is None and index in (1, 2, 3, 4):
-        nominal = {1: 12, 2: 16, 3: 24, 4: 8}[index]
+    if layers is None and index in (1, 2, 3, 4, 5, 6, 7):
+        nominal = {1: 12, 2: 16, 3: 24, 4: 8, 5: 10, 6: 10, 7: 14}[index]
         L = nominal
         # W, state, G resident + ~3 GB for workspace, generator temporaries and the L2 flush buffer
         while L > 1 and synth.resident_bytes(synth.workload(index, L)) + (3 << 30) > free_bytes:
@@ -195,7 +195,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=3, help="parameter set 0..4 (default 3: the ~7B MoE set)")
+    ap.add_argument("--config", type=int, default=3, help="parameter set 0..7 (default 3: the ~7B MoE set; 5-7: the paper's own expert shapes)")
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="mona", choices=["mona", "reference"])
     ap.add_argument("--no-e2e", action="store_true")

@@ -9,7 +9,7 @@ namespace mona {
 
 // A chunk is the unit that goes through prologue -> Newton-Schulz -> update together: up to MAXC
 // same-shape matrices whose bf16 iterates fit the L2 budget.
-constexpr int MAXC = 128;
+constexpr int MAXC = 512;   // the pointer table below travels as a kernel argument (14 KiB of the 32 KiB CUDA 12 allows)
 // Each matrix is cut into at most MAX_SLABS contiguous slabs for the elementwise passes; every slab
 // owns one partial sum of squares, so the Frobenius norm is reduced in a fixed order.
 constexpr int MAX_SLABS = 256;

@@ -31,10 +31,10 @@ namespace {
 constexpr int NSLOTS = 2;
 constexpr size_t WS_STATUS_OFF = 0;
 constexpr size_t WS_CTRL_OFF = 4096;                 // first control block
-constexpr size_t WS_CTRL_BYTES = 256 * 1024;         // per slot
+constexpr size_t WS_CTRL_BYTES = 1024 * 1024;        // per slot
 constexpr size_t CTRL_COUNTERS_OFF = 0;
-constexpr size_t CTRL_INVNORM_OFF = 2048;
-constexpr size_t CTRL_PARTIALS_OFF = 4096;
+constexpr size_t CTRL_INVNORM_OFF = 4096;
+constexpr size_t CTRL_PARTIALS_OFF = 8192;
 constexpr size_t WS_DATA_OFF = WS_CTRL_OFF + NSLOTS * WS_CTRL_BYTES;
 static_assert(CTRL_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS <= WS_CTRL_BYTES, "control block overflow");
 static_assert(sizeof(unsigned int) * MAXC <= CTRL_INVNORM_OFF && sizeof(float) * MAXC <= CTRL_PARTIALS_OFF - CTRL_INVNORM_OFF, "control block overflow");

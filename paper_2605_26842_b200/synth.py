@@ -14,6 +14,12 @@ Parameter sets (the five benchmark configurations):
      4096x4096, bf16 gradients; the layer count is a parameter because the nominal 8 layers
      need more memory than one GPU has.
 
+  5-7  expert matrices of the paper's own models (section "Pretraining"; only the expert shapes are stated,
+     so attention and router weights are left out): 5 = MOE-1B-A0d2B (10 layers, hidden 768, 128 experts of
+     FFN width 256), 6 = MOE-6B-A0d5B (10 layers, hidden 1536, 128 experts of width 1024), 7 = MOE-68B-A3B
+     (14 layers, hidden 3072, 256 experts of width 1024; layer count is a parameter, the full set exceeds
+     one GPU).  Each expert has W1, W3 (width x hidden) and W2 (hidden x width), as in configurations 2-4.
+
 Gradient process per element (stationary AR(1), variance sigma^2, lag-1 correlation rho):
   g_1 = sigma xi_1,   g_k = rho g_{k-1} + sqrt(1 - rho^2) sigma xi_k,
 with xi standard normal, or Student-t with 4 degrees of freedom divided by sqrt(2) (unit variance).
@@ -68,7 +74,7 @@ class Workload:
 
 
 def workload(index: int, layers: int | None = None) -> Workload:
-    """The benchmark configuration `index` (0..4).  `layers` overrides the layer count."""
+    """The benchmark configuration `index` (0..7).  `layers` overrides the layer count."""
     if index == 0:
         return Workload("single_256x512", [MatrixSpec("W", 256, 512)], steps=5, seed=1234)
     if index == 1:
@@ -105,6 +111,16 @@ def workload(index: int, layers: int | None = None) -> Workload:
                       MatrixSpec(f"l{l}.experts.w2", 4096, 1024, 128)]
             specs += [MatrixSpec(f"l{l}.w{q}", 4096, 4096) for q in "qkvo"]
         return Workload(f"moe_shard_{L}L", specs, steps=5, grad_dtype=torch.bfloat16, accel_beta=0.975, seed=1238)
+    if index in (5, 6, 7):
+        nominal, hidden, width, experts, beta = {5: (10, 768, 256, 128, 0.99), 6: (10, 1536, 1024, 128, 0.98),
+                                                  7: (14, 3072, 1024, 256, 0.975)}[index]
+        L = layers or nominal
+        specs = []
+        for l in range(L):
+            specs += [MatrixSpec(f"l{l}.experts.w1", width, hidden, experts), MatrixSpec(f"l{l}.experts.w3", width, hidden, experts),
+                      MatrixSpec(f"l{l}.experts.w2", hidden, width, experts)]
+        name = {5: "paper_moe_1b_experts", 6: "paper_moe_6b_experts", 7: "paper_moe_68b_experts"}[index]
+        return Workload(f"{name}_{L}L", specs, steps=10, accel_beta=beta, seed=1234 + index)
     raise ValueError(f"no such configuration: {index}")
 
 

@@ -100,6 +100,14 @@ def test_mona_lite_state_storage(shapes, grad_dtype, steps):
     assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
 
 
+@pytest.mark.parametrize("shape", [(3, 256, 768), (3, 768, 256), (1, 1024, 1536), (1, 1536, 1024), (1, 1024, 3072),
+                                   (1, 3072, 1024)])
+def test_paper_expert_shapes(shape):
+    """Expert matrices of the paper's three models (FFN width x hidden and its transpose)."""
+    errs = run_case([shape], steps=2, seed=31)
+    check(errs, TOL_O_BF16)
+
+
 def test_plain_muon_path():
     """algorithm = 1: Eq. muon_momentum without the acceleration term; A and G_prev are neither read nor written
     (they stay at their initial zero, so their error against the oracle's untouched zero state is exactly 0)."""
