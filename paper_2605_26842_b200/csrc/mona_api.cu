@@ -278,6 +278,7 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
         if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
     }
     MONA_CUDA(h, tc_gemm_configure(&h->max_pairs));
+    MONA_CUDA(h, small_ns_configure());
     MONA_CUDA(h, cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
     MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
     MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming));
@@ -419,6 +420,14 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                     }
                 }
                 o_final = xb[T & 1];
+            } else if (small_ns_eligible(b.rows, b.cols)) {
+                // short side <= 64 (routers): the whole iteration in one launch, one block per matrix
+                if (phase_mask & 2u) {
+                    MONA_CUDA(h, launch_small_ns(Mc, xf[0], inv_norm, C, (int)b.rows, (int)b.cols, T, ns_a, ns_b, ns_c, stream));
+                    ++h->launches;
+                    h->flops_dense += (double)T * C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
+                }
+                o_final = xf[0];
             } else {
                 if (phase_mask & 2u) {
                     MONA_CUDA(h, launch_scale(Mc, xf[0], inv_norm, C, b.e, b.slab_len, b.slabs, stream));

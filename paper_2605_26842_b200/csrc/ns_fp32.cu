@@ -72,7 +72,138 @@ __global__ void __launch_bounds__(256) sgemm_kernel(SgemmArgs g) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Small matrices (shorter side <= 64, e.g. a 32 x 1024 router): the whole Newton-Schulz iteration of one
+// matrix in ONE block.  The matrix lives in shared memory in its wide orientation Y (s x l, tall inputs
+// are transposed while loading), and every iteration forms A = Y Y^T, B' = b A + c A^2 + a I and
+// Y <- B' Y there, in plain fp32 FMA.  One launch replaces the scale pass and 3T batched SGEMMs, each of
+// which would have had a single block per matrix to work with.
+constexpr int SMALL_THREADS = 256;
+
+template <int SMAX>   // upper bound of the shorter side s: 32 or 64 (register arrays are sized by it)
+__global__ void __launch_bounds__(SMALL_THREADS)
+small_ns_kernel(const float* __restrict__ M, float* __restrict__ O, const float* __restrict__ inv_norm, int rows, int cols,
+                int T, float ca, float cb, float cc) {
+    extern __shared__ float sm[];
+    const bool tall = rows > cols;
+    const int s = tall ? cols : rows, l = tall ? rows : cols;
+    const int lp = l | 1;                 // odd pitch: the transposing load/store of tall inputs stays conflict-free
+    const int sp = s + 1;
+    float* Y = sm;
+    float* A = Y + (size_t)s * lp;
+    float* B = A + s * sp;
+    const long long e = (long long)rows * cols;
+    const float* Mz = M + (long long)blockIdx.x * e;
+    float* Oz = O + (long long)blockIdx.x * e;
+    const float scale = inv_norm[blockIdx.x];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    for (long long idx = tid; idx < e; idx += SMALL_THREADS) {          // X_0 = M / (||M||_F + eps)
+        const int r = (int)(idx / cols), q = (int)(idx - (long long)r * cols);
+        const float v = Mz[idx] * scale;
+        if (!tall) Y[r * lp + q] = v; else Y[q * lp + r] = v;
+    }
+    __syncthreads();
+
+    const int nb = (s + 3) >> 2;          // 4 x 4 blocks of A per side
+    const int nblocks = nb * (nb + 1) / 2;
+    for (int t = 0; t < T; ++t) {
+        // A = Y Y^T: a warp owns a 4 x 4 block on or below the diagonal, its lanes split the l products
+        for (int blk = warp; blk < nblocks; blk += SMALL_THREADS / 32) {
+            int bi = 0;
+            while ((bi + 1) * (bi + 2) / 2 <= blk) ++bi;
+            const int bj = blk - bi * (bi + 1) / 2;
+            float acc[4][4];
+            #pragma unroll
+            for (int r = 0; r < 4; ++r)
+                #pragma unroll
+                for (int q = 0; q < 4; ++q) acc[r][q] = 0.f;
+            for (int k = lane; k < l; k += 32) {
+                float ya[4], yb[4];
+                #pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    ya[r] = (4 * bi + r < s) ? Y[(4 * bi + r) * lp + k] : 0.f;
+                    yb[r] = (4 * bj + r < s) ? Y[(4 * bj + r) * lp + k] : 0.f;
+                }
+                #pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    #pragma unroll
+                    for (int q = 0; q < 4; ++q) acc[r][q] = fmaf(ya[r], yb[q], acc[r][q]);
+            }
+            #pragma unroll
+            for (int r = 0; r < 4; ++r)
+                #pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float v = acc[r][q];
+                    #pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    const int i = 4 * bi + r, j = 4 * bj + q;
+                    if (lane == 0 && i < s && j < s) { A[i * sp + j] = v; A[j * sp + i] = v; }
+                }
+        }
+        __syncthreads();
+        // B' = b A + c A A + a I
+        for (int idx = tid; idx < s * s; idx += SMALL_THREADS) {
+            const int i = idx / s, j = idx - i * s;
+            float sum = 0.f;
+            for (int k = 0; k < s; ++k) sum = fmaf(A[i * sp + k], A[k * sp + j], sum);
+            B[i * sp + j] = fmaf(cb, A[i * sp + j], cc * sum) + (i == j ? ca : 0.f);
+        }
+        __syncthreads();
+        // Y <- B' Y: a thread owns NCOL columns, keeps them in registers and overwrites them in place
+        constexpr int NCOL = SMAX <= 32 ? 4 : 2;
+        for (int c0 = tid * NCOL; c0 < l; c0 += SMALL_THREADS * NCOL) {
+            float y[NCOL][SMAX];
+            #pragma unroll
+            for (int k = 0; k < SMAX; ++k)
+                #pragma unroll
+                for (int u = 0; u < NCOL; ++u) y[u][k] = (k < s && c0 + u < l) ? Y[k * lp + c0 + u] : 0.f;
+            for (int i = 0; i < s; ++i) {
+                float o[NCOL];
+                #pragma unroll
+                for (int u = 0; u < NCOL; ++u) o[u] = 0.f;
+                #pragma unroll
+                for (int k = 0; k < SMAX; ++k) {
+                    const float bik = k < s ? B[i * sp + k] : 0.f;
+                    #pragma unroll
+                    for (int u = 0; u < NCOL; ++u) o[u] = fmaf(bik, y[u][k], o[u]);
+                }
+                #pragma unroll
+                for (int u = 0; u < NCOL; ++u)
+                    if (c0 + u < l) Y[i * lp + c0 + u] = o[u];
+            }
+        }
+        __syncthreads();
+    }
+    for (long long idx = tid; idx < e; idx += SMALL_THREADS) {          // O = X_T, back in the input's orientation
+        const int r = (int)(idx / cols), q = (int)(idx - (long long)r * cols);
+        Oz[idx] = !tall ? Y[r * lp + q] : Y[q * lp + r];
+    }
+}
+
+size_t small_ns_smem(long long s, long long l) { return (size_t)(s * (l | 1) + 2 * s * (s + 1)) * sizeof(float); }
+
 }  // namespace
+
+bool small_ns_eligible(long long rows, long long cols) {
+    const long long s = rows < cols ? rows : cols, l = rows < cols ? cols : rows;
+    return s <= 64 && small_ns_smem(s, l) <= 200 * 1024;
+}
+
+cudaError_t small_ns_configure() {
+    cudaError_t e = cudaFuncSetAttribute(small_ns_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(small_ns_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+}
+
+cudaError_t launch_small_ns(const float* M, float* O, const float* inv_norm, int batch, int rows, int cols, int T,
+                            float a, float b, float c, cudaStream_t stream) {
+    const long long s = rows < cols ? rows : cols, l = rows < cols ? cols : rows;
+    const size_t smem = small_ns_smem(s, l);
+    if (s <= 32) small_ns_kernel<32><<<batch, SMALL_THREADS, smem, stream>>>(M, O, inv_norm, rows, cols, T, a, b, c);
+    else         small_ns_kernel<64><<<batch, SMALL_THREADS, smem, stream>>>(M, O, inv_norm, rows, cols, T, a, b, c);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_sgemm(const SgemmArgs& g, cudaStream_t stream) {
     dim3 grid((g.N + TS - 1) / TS, (g.M + TS - 1) / TS, g.batch);

@@ -16,4 +16,13 @@ struct SgemmArgs {
 };
 cudaError_t launch_sgemm(const SgemmArgs& g, cudaStream_t stream);
 
+// Whole Newton-Schulz iteration (Eq. newton_schulz, T steps, fp32 FMA) of `batch` small matrices, one
+// block per matrix with the matrix resident in shared memory: O = NS_T(M * inv_norm).  M and O are dense
+// [batch][rows][cols].  Only for shapes small_ns_eligible() accepts (shorter side <= 64 and the matrix
+// within 200 KiB of shared memory); call small_ns_configure() once per device first.
+bool small_ns_eligible(long long rows, long long cols);
+cudaError_t small_ns_configure();
+cudaError_t launch_small_ns(const float* M, float* O, const float* inv_norm, int batch, int rows, int cols, int T,
+                            float a, float b, float c, cudaStream_t stream);
+
 }  // namespace mona
