@@ -143,7 +143,11 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp,
 /* End-to-end variant for callers whose gradients arrive in HOST memory: for every descriptor copies
  * grads_host[i] (pinned host memory, same layout and dtype as the device gradient, batch*batch_stride
  * elements) into grads[i], runs the step, and copies the updated parameters back to params_host[i]
- * (pinned, fp32).  Everything is enqueued on `stream`; nothing synchronises. */
+ * (pinned, fp32).  The copies run on two streams the handle owns, pipelined with the step: a chunk starts
+ * as soon as the gradients of its descriptors have arrived, and a descriptor is copied back as soon as its
+ * last matrix is updated, so both transfer directions overlap the computation.  All of it is ordered after
+ * what `stream` held at the call and joined back into `stream` before the call returns; nothing
+ * synchronises the host. */
 mona_status mona_step_host(mona_handle* h, const mona_hparams* hp,
                            void* const* params, void* const* grads,
                            const void* const* grads_host, void* const* params_host, void* stream);

@@ -183,6 +183,11 @@ struct mona_handle {
     uint8_t* ws = nullptr;
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // host-to-host pipeline of mona_step_host(): copy streams and per-descriptor events, created on first use
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev_hfork = nullptr, ev_hjoin = nullptr;
+    std::vector<cudaEvent_t> ev_in;     // gradient of descriptor i has arrived on the device
+    std::vector<cudaEvent_t> ev_out;    // 2 per descriptor: its chunks on slot stream 0 / 1 have been updated
     DeviceStatus* host_status = nullptr;   // pinned
     std::string last_error;
     int64_t launches = 0;
@@ -292,8 +297,13 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
     return MONA_OK;
 }
 
-mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads,
-                         void* const* o_out, uint32_t phase_mask, void* stream_v) {
+}  // extern "C"
+
+// One optimizer step.  With `params_host` set (mona_step_host) every chunk first waits for the gradient copies of
+// the descriptors it touches, and a descriptor whose last matrix has been updated is copied back right away
+// on the handle's device-to-host stream, so transfers in both directions overlap the remaining chunks.
+static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads,
+                             void* const* o_out, uint32_t phase_mask, void* stream_v, void* const* params_host) {
     if (!h) return MONA_ERR_INVALID_ARG;
     if (!hp || !params || !grads) return h->fail(MONA_ERR_INVALID_ARG, "hp, params or grads is null");
     if (hp->ns_steps < 0 || hp->ns_steps > 64) return h->fail(MONA_ERR_INVALID_ARG, "ns_steps out of range");
@@ -334,6 +344,8 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
         MONA_CUDA(h, cudaStreamWaitEvent(h->side, h->ev_fork, 0));
     }
     int64_t chunk_index = 0;
+    std::vector<char> out_recorded(params_host ? 2 * plan.descs.size() : 0, 0);
+    std::vector<int> chunk_descs;
     h->launches = 0;
     h->flops_exec = 0.0;
     h->flops_dense = 0.0;
@@ -352,9 +364,11 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             const int C = (int)std::min<int64_t>(cap, count - start);
             ChunkPtrs ptrs;
             bool vec4 = (b.e % 4 == 0);
+            chunk_descs.clear();
             for (int c = 0; c < C; ++c) {
                 const MatRef& mr = b.mats[start + c];
                 const mona_matrix_desc& d = plan.descs[mr.desc];
+                if (chunk_descs.empty() || chunk_descs.back() != mr.desc) chunk_descs.push_back(mr.desc);
                 if ((d.batch_stride * (int64_t)gsz) % 16 != 0 || (d.batch_stride * 4) % 16 != 0) vec4 = false;
                 ptrs.g[c] = (const uint8_t*)grads[mr.desc] + (size_t)mr.b * d.batch_stride * gsz;
                 ptrs.w[c] = (float*)params[mr.desc] + mr.b * d.batch_stride;
@@ -378,6 +392,8 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
             float* af = (float*)(data + b.off32_a);
             float* bf = (float*)(data + b.off32_b);
 
+            if (params_host)
+                for (int dsc : chunk_descs) MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_in[dsc], 0));
             if (phase_mask & 1u) {
                 MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16,
                                              hp->algorithm == 1 ? PROLOGUE_NO_AUX : (b.state_dtype == MONA_BF16 ? PROLOGUE_AUX_BF16 : PROLOGUE_AUX_F32), vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
@@ -470,6 +486,21 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
                 MONA_CUDA(h, launch_update(ptrs, C, tc, vec4, o_final, b.e, b.slab_len, b.slabs, eta_lambda, eta_gamma, stream));
                 ++h->launches;
             }
+            if (params_host) {
+                for (int dsc : chunk_descs) {
+                    MONA_CUDA(h, cudaEventRecord(h->ev_out[2 * dsc + slot], stream));
+                    out_recorded[2 * dsc + slot] = 1;
+                }
+                const MatRef& last = b.mats[start + C - 1];
+                for (int dsc : chunk_descs) {
+                    const mona_matrix_desc& d = plan.descs[dsc];
+                    if (dsc == last.desc && last.b != d.batch - 1) continue;    // descriptor continues in the next chunk
+                    for (int sl = 0; sl < NSLOTS; ++sl)
+                        if (out_recorded[2 * dsc + sl]) MONA_CUDA(h, cudaStreamWaitEvent(h->d2h, h->ev_out[2 * dsc + sl], 0));
+                    const size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * 4;
+                    MONA_CUDA(h, cudaMemcpyAsync(params_host[dsc], params[dsc], bytes, cudaMemcpyDeviceToHost, h->d2h));
+                }
+            }
         }
     }
     if (overlap) {
@@ -479,8 +510,15 @@ mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* pa
     return MONA_OK;
 }
 
+extern "C" {
+
+mona_status mona_step_ex(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads,
+                         void* const* o_out, uint32_t phase_mask, void* stream_v) {
+    return step_impl(h, hp, params, grads, o_out, phase_mask, stream_v, nullptr);
+}
+
 mona_status mona_step(mona_handle* h, const mona_hparams* hp, void* const* params, const void* const* grads, void* stream) {
-    return mona_step_ex(h, hp, params, grads, nullptr, 7u, stream);
+    return step_impl(h, hp, params, grads, nullptr, 7u, stream, nullptr);
 }
 
 mona_status mona_step_host(mona_handle* h, const mona_hparams* hp, void* const* params, void* const* grads,
@@ -490,20 +528,39 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp, void* const* 
     cudaStream_t stream = (cudaStream_t)stream_v;
     MONA_CUDA(h, cudaSetDevice(h->device));
     const int64_t n_desc = (int64_t)h->plan.descs.size();
-    for (int64_t i = 0; i < n_desc; ++i) {
-        const mona_matrix_desc& d = h->plan.descs[i];
-        if (!grads_host[i] || !grads[i]) return h->fail(MONA_ERR_INVALID_ARG, "grads_host[%lld] or grads[%lld] is null", (long long)i, (long long)i);
-        size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * (d.grad_dtype == MONA_BF16 ? 2 : 4);
-        MONA_CUDA(h, cudaMemcpyAsync(grads[i], grads_host[i], bytes, cudaMemcpyHostToDevice, stream));
+    for (int64_t i = 0; i < n_desc; ++i)
+        if (!grads_host[i] || !grads[i] || !params_host[i] || !params[i])
+            return h->fail(MONA_ERR_INVALID_ARG, "descriptor %lld: a gradient or parameter pointer (host or device) is null", (long long)i);
+    if (!h->h2d) {
+        MONA_CUDA(h, cudaStreamCreateWithFlags(&h->h2d, cudaStreamNonBlocking));
+        MONA_CUDA(h, cudaStreamCreateWithFlags(&h->d2h, cudaStreamNonBlocking));
+        MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_hfork, cudaEventDisableTiming));
+        MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_hjoin, cudaEventDisableTiming));
+        h->ev_in.assign((size_t)n_desc, nullptr);
+        h->ev_out.assign((size_t)(2 * n_desc), nullptr);
+        for (auto& e : h->ev_in) MONA_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        for (auto& e : h->ev_out) MONA_CUDA(h, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     }
-    mona_status st = mona_step_ex(h, hp, params, (const void* const*)grads, nullptr, 7u, stream_v);
+    // both copy streams start after whatever the caller's stream holds so far
+    MONA_CUDA(h, cudaEventRecord(h->ev_hfork, stream));
+    MONA_CUDA(h, cudaStreamWaitEvent(h->h2d, h->ev_hfork, 0));
+    MONA_CUDA(h, cudaStreamWaitEvent(h->d2h, h->ev_hfork, 0));
+    // gradients travel in the order in which the chunks will want them: bucket by bucket, descriptor by descriptor
+    for (const Bucket& b : h->plan.buckets) {
+        int prev = -1;
+        for (const MatRef& mr : b.mats) {
+            if (mr.desc == prev) continue;
+            prev = mr.desc;
+            const mona_matrix_desc& d = h->plan.descs[mr.desc];
+            const size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * (d.grad_dtype == MONA_BF16 ? 2 : 4);
+            MONA_CUDA(h, cudaMemcpyAsync(grads[mr.desc], grads_host[mr.desc], bytes, cudaMemcpyHostToDevice, h->h2d));
+            MONA_CUDA(h, cudaEventRecord(h->ev_in[mr.desc], h->h2d));
+        }
+    }
+    mona_status st = step_impl(h, hp, params, (const void* const*)grads, nullptr, 7u, stream_v, params_host);
     if (st != MONA_OK) return st;
-    for (int64_t i = 0; i < n_desc; ++i) {
-        const mona_matrix_desc& d = h->plan.descs[i];
-        if (!params_host[i]) return h->fail(MONA_ERR_INVALID_ARG, "params_host[%lld] is null", (long long)i);
-        size_t bytes = (size_t)((d.batch - 1) * d.batch_stride + d.rows * d.cols) * 4;
-        MONA_CUDA(h, cudaMemcpyAsync(params_host[i], params[i], bytes, cudaMemcpyDeviceToHost, stream));
-    }
+    MONA_CUDA(h, cudaEventRecord(h->ev_hjoin, h->d2h));
+    MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_hjoin, 0));
     return MONA_OK;
 }
 
@@ -548,6 +605,12 @@ void mona_destroy(mona_handle* h) {
     if (!h) return;
     if (h->side) cudaStreamDestroy(h->side);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->h2d) cudaStreamDestroy(h->h2d);
+    if (h->d2h) cudaStreamDestroy(h->d2h);
+    if (h->ev_hfork) cudaEventDestroy(h->ev_hfork);
+    if (h->ev_hjoin) cudaEventDestroy(h->ev_hjoin);
+    for (cudaEvent_t e : h->ev_in) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : h->ev_out) if (e) cudaEventDestroy(e);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->host_status) cudaFreeHost(h->host_status);
     delete h;

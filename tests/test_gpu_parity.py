@@ -177,3 +177,43 @@ def test_deterministic_and_resumable():
     a, b, c = run(False), run(False), run(True)
     for x, y, z in zip(a, b, c):
         assert torch.equal(x, y) and torch.equal(x, z)
+
+
+def test_step_host_matches_step_and_returns_parameters():
+    """mona_step_host (pinned host gradients in, parameters out, transfers pipelined with the chunks) gives
+    bit-identical parameters and state to mona_step on the same inputs, and the host copy equals the device's.
+    A small chunk budget makes descriptors straddle chunks and both workspace slots take part."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(77)
+    shapes = [(5, 256, 384), (5, 256, 384), (3, 384, 256), (1, 32, 256)]
+    W0 = [torch.randn(s, generator=gen) * 0.02 for s in shapes]
+    G = [[torch.randn(s, generator=gen) * 1e-3 for s in shapes] for _ in range(3)]
+    hp = pkg.default_hparams()
+    pkg.set_chunk_budget(2 << 20)            # 3 matrices of 256x384 per chunk
+    try:
+        def run(host):
+            p = [w.clone().to(dev) for w in W0]
+            opt = pkg.MonaOptimizer(p)
+            g_dev = [torch.zeros_like(w, device=dev) for w in W0]
+            g_host = [torch.empty(s, pin_memory=True) for s in shapes]
+            p_host = [torch.zeros(s, pin_memory=True) for s in shapes]
+            for k in range(3):
+                if host:
+                    for h_, g in zip(g_host, G[k]):
+                        h_.copy_(g)
+                    opt.step_host(hp, p, g_dev, g_host, p_host)
+                    torch.cuda.synchronize()
+                    for ph, pd in zip(p_host, p):
+                        assert torch.equal(ph, pd.cpu())
+                else:
+                    opt.step(hp, p, [g.to(dev) for g in G[k]])
+            torch.cuda.synchronize()
+            assert opt.poll_status()[0] == 0
+            out = [t.clone() for t in p] + [opt.state.clone()]
+            opt.close()
+            return out
+        a, b = run(False), run(True)
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    finally:
+        pkg.set_chunk_budget(768 << 20)
