@@ -217,3 +217,32 @@ def test_step_host_matches_step_and_returns_parameters():
             assert torch.equal(x, y)
     finally:
         pkg.set_chunk_budget(768 << 20)
+
+
+def test_chunk_overlap_does_not_change_results():
+    """Two chunks in flight on two streams (default) and everything on the caller's stream give bit-identical
+    parameters and state."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(9)
+    shapes = [(7, 256, 384), (2, 384, 256), (1, 512, 512)]
+    W0 = [torch.randn(s, generator=gen) * 0.02 for s in shapes]
+    G = [[torch.randn(s, generator=gen) * 1e-3 for s in shapes] for _ in range(3)]
+    hp = pkg.default_hparams()
+    pkg.set_chunk_budget(2 << 20)
+    try:
+        def run(overlap):
+            pkg.set_chunk_overlap(overlap)
+            p = [w.clone().to(dev) for w in W0]
+            opt = pkg.MonaOptimizer(p)
+            for k in range(3):
+                opt.step(hp, p, [g.to(dev) for g in G[k]])
+            torch.cuda.synchronize()
+            out = [t.clone() for t in p] + [opt.state.clone()]
+            opt.close()
+            return out
+        a, b = run(True), run(False)
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    finally:
+        pkg.set_chunk_overlap(True)
+        pkg.set_chunk_budget(768 << 20)
