@@ -203,6 +203,7 @@ def main():
     ap.add_argument("--chunk-mb", type=int, default=None, help="override the chunk budget (MiB)")
     ap.add_argument("--no-overlap", action="store_true", help="keep all chunks on one stream")
     ap.add_argument("--muon", action="store_true", help="plain Muon step (no acceleration term): the baseline of the paper's timing claim")
+    ap.add_argument("--single-buffer", action="store_true", help="state kept as M and Z = beta_a A - (1 - beta_a) G (one fp32 buffer instead of A and G_prev)")
     ap.add_argument("--lite", action="store_true", help="MONA-Lite storage: A_k and G_{k-1} kept in bfloat16")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -232,7 +233,7 @@ def main():
     params = synth.init_params(wl, dev, seed_offset=rank)
     gp = synth.GradientProcess(wl, dev, keep_fp32_shadow=False)
     opt = pkg.MonaOptimizer(params, grad_dtype=wl.grad_dtype, device=local_rank,
-                            state_dtype=torch.bfloat16 if args.lite else torch.float32)
+                            state_dtype=pkg.MONA_STATE_COMBINED if args.single_buffer else (torch.bfloat16 if args.lite else torch.float32))
     hp = pkg.default_hparams(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha, algorithm=1 if args.muon else 0)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
@@ -295,6 +296,8 @@ def main():
     peaks, peak_src = load_peaks()
     n = wl.n_params
     pro_elem = g_elem + 2 * aux + 4 + 2 * aux + 4 + 2   # read G, G_prev, A, M; write G_prev, A, M, bf16 X
+    if args.single_buffer:
+        pro_elem = g_elem + 4 + 4 + 4 + 4 + 2           # read G, Z, M; write Z, M, bf16 X
     if args.muon:
         pro_elem = g_elem + 4 + 4 + 2                   # read G, M; write M, bf16 X
     pro_bytes = n * pro_elem
@@ -359,7 +362,7 @@ def main():
                            "grad_dtype": str(wl.grad_dtype).replace("torch.", ""), "gradient_process":
                            f"AR(1) rho={wl.rho} sigma={wl.sigma} {wl.dist}", "ns_steps": hp.ns_steps,
                            "accel_beta": wl.accel_beta, "accel_alpha": wl.accel_alpha,
-                           "state_storage": "bf16 A_k and G_{k-1} (MONA-Lite)" if args.lite else "fp32",
+                           "state_storage": "single fp32 buffer Z" if args.single_buffer else ("bf16 A_k and G_{k-1} (MONA-Lite)" if args.lite else "fp32"),
                            "algorithm": "Muon (no acceleration term)" if args.muon else "MONA", "parallelism":
                            "independent parameter set per GPU, no collective" if world > 1 else "single GPU",
                            "l2": "inputs larger than L2 and a 256 MiB buffer rewritten between timed steps",

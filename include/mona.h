@@ -51,6 +51,8 @@ typedef enum {
 } mona_status;
 
 typedef enum { MONA_F32 = 0, MONA_BF16 = 1 } mona_dtype;
+/* Third value of mona_matrix_desc.state_dtype (see there). */
+#define MONA_STATE_COMBINED 2
 
 /* One descriptor = `batch` matrices of identical shape (the experts of one MoE layer, or batch = 1).
  * Matrix b of the descriptor starts `b * batch_stride` ELEMENTS after the descriptor's base pointer,
@@ -66,7 +68,14 @@ typedef struct {
                                   Deployment with Reduced Overhead"): both buffers kept in bfloat16, equations
                                   unchanged.  A_k is formed in fp32, rounded to nearest-even once when stored,
                                   and the stored value is the one G~_k uses; G_{k-1} is the rounded G_k.
-                                  M_k is fp32 either way.                                              */
+                                  M_k is fp32 either way.
+                                  MONA_STATE_COMBINED (2): one fp32 buffer Z_k = beta_a A_k - (1-beta_a) G_k in
+                                  place of both.  A_k and G_{k-1} enter the next step only through it
+                                  (A_{k+1} = Z_k + (1-beta_a) G_{k+1}), so the step is Algorithm 1 unchanged with
+                                  8 instead of 12 state bytes per parameter and 22 instead of 30 bytes moved by
+                                  the prologue - the counterpart, at this boundary, of the paper's "streaming"
+                                  variant that drops the G_{k-1} buffer.  mona_state_layout() then reports Z at
+                                  off_A and (size_t)-1 for off_Gprev.                                  */
 } mona_matrix_desc;
 
 /* REQUIRE line of Algorithm 1.  Doubles on purpose: (1 - beta_a), eta*gamma and eta*lambda are formed

@@ -14,6 +14,7 @@ STATUS_NAMES = {0: "MONA_OK", 1: "MONA_ERR_INVALID_ARG", 2: "MONA_ERR_UNSUPPORTE
                 4: "MONA_ERR_CUDA", 5: "MONA_ERR_TIMEOUT", 6: "MONA_ERR_NONFINITE", 7: "MONA_ERR_ARCH",
                 8: "MONA_ERR_BUFFER_TOO_SMALL"}
 MONA_F32, MONA_BF16 = 0, 1
+MONA_STATE_COMBINED = 2      # single auxiliary buffer Z = beta_a A - (1 - beta_a) G
 
 
 class MonaError(RuntimeError):
@@ -134,7 +135,8 @@ class MonaOptimizer:
             batch = p.shape[0] if p.dim() == 3 else 1
             rows, cols = p.shape[-2], p.shape[-1]
             self.descs.append(MatrixDesc(rows, cols, batch, rows * cols, MONA_BF16 if grad_dtype == torch.bfloat16 else MONA_F32,
-                                         MONA_BF16 if state_dtype == torch.bfloat16 else MONA_F32))
+                                         state_dtype if isinstance(state_dtype, int) else
+                                         (MONA_BF16 if state_dtype == torch.bfloat16 else MONA_F32)))
         self.device = torch.cuda.current_device() if device is None else device
         self.grad_dtype = grad_dtype
         sb, wb = query_sizes(self.descs)
@@ -184,13 +186,17 @@ class MonaOptimizer:
 
     def state_views(self, desc: int):
         """Views (batch, rows, cols) of M, A, G_prev of descriptor `desc` inside the state block: M fp32,
-        A and G_prev in the descriptor's state dtype."""
+        A and G_prev in the descriptor's state dtype.  In the single-buffer format the second view is Z and
+        the third is None."""
         d = self.descs[desc]
         n = d.batch * d.rows * d.cols
         aux = torch.bfloat16 if d.state_dtype == MONA_BF16 else torch.float32
         offs = self.state_layout(desc)
         out = []
         for off, dt in zip(offs, (torch.float32, aux, aux)):
+            if off == C.c_size_t(-1).value:
+                out.append(None)
+                continue
             sz = 2 if dt == torch.bfloat16 else 4
             out.append(self.state[off: off + n * sz].view(dt).view(d.batch, d.rows, d.cols))
         return tuple(out)

@@ -43,6 +43,8 @@ template <typename ST>
 struct StateIO;
 template <>
 struct StateIO<float> {
+    using elem = float;
+    static constexpr bool has_gp = true;
     static __device__ __forceinline__ float4 load4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
     static __device__ __forceinline__ void store4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
     static __device__ __forceinline__ float load1(const float* p) { return *p; }
@@ -51,6 +53,8 @@ struct StateIO<float> {
 };
 template <>
 struct StateIO<__nv_bfloat16> {
+    using elem = __nv_bfloat16;
+    static constexpr bool has_gp = true;
     static __device__ __forceinline__ float4 load4(const __nv_bfloat16* p) { return GradLoad<__nv_bfloat16>::load4(p); }
     static __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {     // v holds already-rounded values
         __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
@@ -61,16 +65,45 @@ struct StateIO<__nv_bfloat16> {
     static __device__ __forceinline__ float round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 };
 
+// Tag for the single-buffer ("streaming") form of the acceleration state.  A_k and G_{k-1} enter step k+1 only
+// through Z_k = beta_a A_k - (1 - beta_a) G_k:  A_{k+1} = beta_a A_k + (1 - beta_a)(G_{k+1} - G_k) = Z_k + (1 - beta_a) G_{k+1}.
+// So one fp32 buffer Z replaces the two of Algorithm 1 (Z_0 = 0), and the pass moves 22 bytes per element, not 30.
+// The buffer travels through the kernel in the `A` slot; the `G_prev` slot is unused.
+struct Combined {};
+template <>
+struct StateIO<Combined> : StateIO<float> {
+    static constexpr bool has_gp = false;
+};
+
 // Tag for the plain Muon step (Eq. muon_momentum): there is no acceleration state to read or write.
 struct NoAux {};
 template <>
 struct StateIO<NoAux> {
-    static __device__ __forceinline__ float4 load4(const NoAux*) { return make_float4(0.f, 0.f, 0.f, 0.f); }
-    static __device__ __forceinline__ void store4(NoAux*, float4) {}
-    static __device__ __forceinline__ float load1(const NoAux*) { return 0.f; }
-    static __device__ __forceinline__ void store1(NoAux*, float) {}
+    using elem = float;
+    static constexpr bool has_gp = false;
+    static __device__ __forceinline__ float4 load4(const float*) { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ void store4(float*, float4) {}
+    static __device__ __forceinline__ float load1(const float*) { return 0.f; }
+    static __device__ __forceinline__ void store1(float*, float) {}
     static __device__ __forceinline__ float round(float v) { return v; }
 };
+// The G_{k-1} slot only exists in the two-buffer formats.
+template <typename ST>
+__device__ __forceinline__ float4 gp_load4(const typename StateIO<ST>::elem* p) {
+    if constexpr (StateIO<ST>::has_gp) return StateIO<ST>::load4(p); else return make_float4(0.f, 0.f, 0.f, 0.f);
+}
+template <typename ST>
+__device__ __forceinline__ void gp_store4(typename StateIO<ST>::elem* p, float4 v) {
+    if constexpr (StateIO<ST>::has_gp) StateIO<ST>::store4(p, v);
+}
+template <typename ST>
+__device__ __forceinline__ float gp_load1(const typename StateIO<ST>::elem* p) {
+    if constexpr (StateIO<ST>::has_gp) return StateIO<ST>::load1(p); else return 0.f;
+}
+template <typename ST>
+__device__ __forceinline__ void gp_store1(typename StateIO<ST>::elem* p, float v) {
+    if constexpr (StateIO<ST>::has_gp) StateIO<ST>::store1(p, v);
+}
 
 template <typename ST>
 __device__ __forceinline__ void mona_elem(float g, float& gp, float& a, float& m, const PrologueScalars& k) {
@@ -80,6 +113,15 @@ __device__ __forceinline__ void mona_elem(float g, float& gp, float& a, float& m
     float gt = mul_add2(k.alpha, a, g);                             // G~_k = G_k + alpha A_k
     m = mul_add2(k.mu, m, gt);                                      // M_k = mu M_{k-1} + G~_k
     gp = StateIO<ST>::round(g);                                     // G_{k-1} <- G_k
+}
+template <>
+__device__ __forceinline__ void mona_elem<Combined>(float g, float&, float& z, float& m, const PrologueScalars& k) {
+    const float w = fmaf(k.one_minus_beta.hi, g, k.one_minus_beta.lo * g);   // (1 - beta_a) G_k
+    const float a = z + w;                                          // A_k = Z_{k-1} + (1 - beta_a) G_k
+    float gt = mul_add2(k.alpha, a, g);                             // G~_k = G_k + alpha A_k
+    m = mul_add2(k.mu, m, gt);                                      // M_k = mu M_{k-1} + G~_k
+    // Z_k = beta_a A_k - (1 - beta_a) G_k = beta_a Z_{k-1} - (1 - beta_a)^2 G_k; the second form does not cancel
+    z = mul_add2(k.beta, z, -fmaf(k.one_minus_beta.hi, w, k.one_minus_beta.lo * w));
 }
 template <>
 __device__ __forceinline__ void mona_elem<NoAux>(float g, float&, float&, float& m, const PrologueScalars& k) {
@@ -111,7 +153,7 @@ __device__ __forceinline__ float block_sum(float v, float* smem /* >= 8 floats *
 // depend on scheduling; it then resets the arrival counter for the next call.
 template <typename GT, typename ST, int VEC>
 __global__ void __launch_bounds__(EW_THREADS)
-prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, ST* __restrict__ Gpst,
+prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, void* __restrict__ Ast, void* __restrict__ Gpst,
                 __nv_bfloat16* __restrict__ xhat, float* __restrict__ partials, unsigned int* __restrict__ counters,
                 float* __restrict__ inv_norm, DeviceStatus* __restrict__ status, long long e, long long slab_len,
                 int slabs, PrologueScalars k) {
@@ -122,8 +164,9 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, S
     const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
     const GT* __restrict__ g = reinterpret_cast<const GT*>(ptrs.g[c]);
     float* __restrict__ M = Mst + (long long)c * e;
-    ST* __restrict__ A = Ast ? Ast + (long long)c * e : nullptr;      // pointer arithmetic only; NoAux never dereferences
-    ST* __restrict__ Gp = Gpst ? Gpst + (long long)c * e : nullptr;
+    using AuxT = typename StateIO<ST>::elem;
+    AuxT* __restrict__ A = reinterpret_cast<AuxT*>(Ast) + (long long)c * e;      // never dereferenced by formats without it
+    AuxT* __restrict__ Gp = reinterpret_cast<AuxT*>(Gpst) + (long long)c * e;
     __nv_bfloat16* __restrict__ X = xhat ? xhat + (long long)c * e : nullptr;
 
     float acc = 0.f;
@@ -133,14 +176,14 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, S
         // two independent vectors per trip keep ~128 B per thread in flight
         for (; i + STEP < hi; i += 2 * STEP) {
             float4 g0 = GradLoad<GT>::load4(g + i), g1 = GradLoad<GT>::load4(g + i + STEP);
-            float4 p0 = StateIO<ST>::load4(Gp + i), p1 = StateIO<ST>::load4(Gp + i + STEP);
+            float4 p0 = gp_load4<ST>(Gp + i), p1 = gp_load4<ST>(Gp + i + STEP);
             float4 a0 = StateIO<ST>::load4(A + i), a1 = StateIO<ST>::load4(A + i + STEP);
             float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i)), m1 = __ldcs(reinterpret_cast<const float4*>(M + i + STEP));
             mona_elem<ST>(g0.x, p0.x, a0.x, m0.x, k); mona_elem<ST>(g0.y, p0.y, a0.y, m0.y, k);
             mona_elem<ST>(g0.z, p0.z, a0.z, m0.z, k); mona_elem<ST>(g0.w, p0.w, a0.w, m0.w, k);
             mona_elem<ST>(g1.x, p1.x, a1.x, m1.x, k); mona_elem<ST>(g1.y, p1.y, a1.y, m1.y, k);
             mona_elem<ST>(g1.z, p1.z, a1.z, m1.z, k); mona_elem<ST>(g1.w, p1.w, a1.w, m1.w, k);
-            StateIO<ST>::store4(Gp + i, p0); StateIO<ST>::store4(Gp + i + STEP, p1);
+            gp_store4<ST>(Gp + i, p0); gp_store4<ST>(Gp + i + STEP, p1);
             StateIO<ST>::store4(A + i, a0);  StateIO<ST>::store4(A + i + STEP, a1);
             __stcs(reinterpret_cast<float4*>(M + i), m0);  __stcs(reinterpret_cast<float4*>(M + i + STEP), m1);
             if (X) {
@@ -152,12 +195,12 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, S
         }
         for (; i < hi; i += STEP) {
             float4 g0 = GradLoad<GT>::load4(g + i);
-            float4 p0 = StateIO<ST>::load4(Gp + i);
+            float4 p0 = gp_load4<ST>(Gp + i);
             float4 a0 = StateIO<ST>::load4(A + i);
             float4 m0 = __ldcs(reinterpret_cast<const float4*>(M + i));
             mona_elem<ST>(g0.x, p0.x, a0.x, m0.x, k); mona_elem<ST>(g0.y, p0.y, a0.y, m0.y, k);
             mona_elem<ST>(g0.z, p0.z, a0.z, m0.z, k); mona_elem<ST>(g0.w, p0.w, a0.w, m0.w, k);
-            StateIO<ST>::store4(Gp + i, p0);
+            gp_store4<ST>(Gp + i, p0);
             StateIO<ST>::store4(A + i, a0);
             __stcs(reinterpret_cast<float4*>(M + i), m0);
             if (X) *reinterpret_cast<uint2*>(X + i) = make_uint2(pack_bf16x2(m0.x, m0.y), pack_bf16x2(m0.z, m0.w));
@@ -165,9 +208,9 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, ST* __restrict__ Ast, S
         }
     } else {
         for (long long i = lo + threadIdx.x; i < hi; i += EW_THREADS) {
-            float gv = GradLoad<GT>::load1(g + i), pv = StateIO<ST>::load1(Gp + i), av = StateIO<ST>::load1(A + i), mv = M[i];
+            float gv = GradLoad<GT>::load1(g + i), pv = gp_load1<ST>(Gp + i), av = StateIO<ST>::load1(A + i), mv = M[i];
             mona_elem<ST>(gv, pv, av, mv, k);
-            StateIO<ST>::store1(Gp + i, pv); StateIO<ST>::store1(A + i, av); M[i] = mv;
+            gp_store1<ST>(Gp + i, pv); StateIO<ST>::store1(A + i, av); M[i] = mv;
             if (X) X[i] = __float2bfloat16_rn(mv);
             acc = fmaf(mv, mv, acc);
         }
@@ -248,8 +291,8 @@ template <typename GT, typename ST>
 void launch_prologue_t(dim3 grid, dim3 block, cudaStream_t stream, bool vec4, const ChunkPtrs& ptrs, float* M, void* A, void* Gp,
                        __nv_bfloat16* xhat, float* partials, unsigned int* counters, float* inv_norm, DeviceStatus* status,
                        long long e, long long slab_len, int slabs, const PrologueScalars& k) {
-    if (vec4) prologue_kernel<GT, ST, 4><<<grid, block, 0, stream>>>(ptrs, M, (ST*)A, (ST*)Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
-    else      prologue_kernel<GT, ST, 1><<<grid, block, 0, stream>>>(ptrs, M, (ST*)A, (ST*)Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+    if (vec4) prologue_kernel<GT, ST, 4><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
+    else      prologue_kernel<GT, ST, 1><<<grid, block, 0, stream>>>(ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k);
 }
 }  // namespace
 
@@ -261,10 +304,12 @@ cudaError_t launch_prologue(const ChunkPtrs& ptrs, int C, bool grad_bf16, int st
 #define MONA_PROLOGUE_CASE(GT, ST) launch_prologue_t<GT, ST>(grid, block, stream, vec4, ptrs, M, A, Gp, xhat, partials, counters, inv_norm, status, e, slab_len, slabs, k)
     if (grad_bf16) {
         if (state_kind == PROLOGUE_NO_AUX) MONA_PROLOGUE_CASE(__nv_bfloat16, NoAux);
+        else if (state_kind == PROLOGUE_AUX_COMBINED) MONA_PROLOGUE_CASE(__nv_bfloat16, Combined);
         else if (state_kind == PROLOGUE_AUX_BF16) MONA_PROLOGUE_CASE(__nv_bfloat16, __nv_bfloat16);
         else MONA_PROLOGUE_CASE(__nv_bfloat16, float);
     } else {
         if (state_kind == PROLOGUE_NO_AUX) MONA_PROLOGUE_CASE(float, NoAux);
+        else if (state_kind == PROLOGUE_AUX_COMBINED) MONA_PROLOGUE_CASE(float, Combined);
         else if (state_kind == PROLOGUE_AUX_BF16) MONA_PROLOGUE_CASE(float, __nv_bfloat16);
         else MONA_PROLOGUE_CASE(float, float);
     }

@@ -89,7 +89,7 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         mona_matrix_desc& d = plan.descs[i];
         if (d.rows <= 0 || d.cols <= 0 || d.batch <= 0) { err = "descriptor with non-positive rows/cols/batch"; return MONA_ERR_INVALID_ARG; }
         if (d.grad_dtype != MONA_F32 && d.grad_dtype != MONA_BF16) { err = "descriptor with unknown grad_dtype"; return MONA_ERR_INVALID_ARG; }
-        if (d.state_dtype != MONA_F32 && d.state_dtype != MONA_BF16) { err = "descriptor with unknown state_dtype"; return MONA_ERR_INVALID_ARG; }
+        if (d.state_dtype != MONA_F32 && d.state_dtype != MONA_BF16 && d.state_dtype != MONA_STATE_COMBINED) { err = "descriptor with unknown state_dtype"; return MONA_ERR_INVALID_ARG; }
         if (d.rows > (1 << 20) || d.cols > (1 << 20) || d.rows * d.cols > (1ll << 31)) { err = "matrix too large"; return MONA_ERR_UNSUPPORTED_SHAPE; }
         if (d.batch_stride == 0) d.batch_stride = d.rows * d.cols;
         if (d.batch_stride < d.rows * d.cols) { err = "batch_stride smaller than rows*cols"; return MONA_ERR_INVALID_ARG; }
@@ -123,7 +123,8 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         const size_t aux = b.state_dtype == MONA_BF16 ? 2 : 4;              // every block starts 256-byte aligned
         b.off_M = state_bytes; state_bytes += align_up((size_t)count * b.e * 4, 256);
         b.off_A = state_bytes; state_bytes += align_up((size_t)count * b.e * aux, 256);
-        b.off_G = state_bytes; state_bytes += align_up((size_t)count * b.e * aux, 256);
+        b.off_G = state_bytes;                                              // the single-buffer form has no G_prev block
+        if (b.state_dtype != MONA_STATE_COMBINED) state_bytes += align_up((size_t)count * b.e * aux, 256);
         // slabs: ~16K elements each, at most MAX_SLABS, slab length a multiple of 1024
         int64_t slab = 16384;
         if ((b.e + slab - 1) / slab > MAX_SLABS) slab = (int64_t)align_up((size_t)((b.e + MAX_SLABS - 1) / MAX_SLABS), 1024);
@@ -396,7 +397,8 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                 for (int dsc : chunk_descs) MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_in[dsc], 0));
             if (phase_mask & 1u) {
                 MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16,
-                                             hp->algorithm == 1 ? PROLOGUE_NO_AUX : (b.state_dtype == MONA_BF16 ? PROLOGUE_AUX_BF16 : PROLOGUE_AUX_F32), vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
+                                             hp->algorithm == 1 ? PROLOGUE_NO_AUX : (b.state_dtype == MONA_BF16 ? PROLOGUE_AUX_BF16 :
+                                                 b.state_dtype == MONA_STATE_COMBINED ? PROLOGUE_AUX_COMBINED : PROLOGUE_AUX_F32), vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
                                              counters, inv_norm, dstatus, b.e, b.slab_len, b.slabs, ps, stream));
                 ++h->launches;
             }
@@ -586,7 +588,7 @@ mona_status mona_state_layout(const mona_handle* h, int64_t desc, size_t* off_M,
     const size_t pos = (size_t)h->plan.desc_pos[desc] * (size_t)b.e;
     if (off_M) *off_M = b.off_M + pos * 4;
     if (off_A) *off_A = b.off_A + pos * aux;
-    if (off_Gprev) *off_Gprev = b.off_G + pos * aux;
+    if (off_Gprev) *off_Gprev = b.state_dtype == MONA_STATE_COMBINED ? (size_t)-1 : b.off_G + pos * aux;
     return MONA_OK;
 }
 

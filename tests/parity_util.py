@@ -59,7 +59,7 @@ def ar1_grads(shapes, steps, rho, sigma, seed, dtype=torch.float32, heavy_tail=F
 
 
 def run_case(shapes, steps=3, hp=None, grad_dtype=torch.float32, rho=0.9, sigma=1e-3, seed=0, heavy_tail=False,
-             pad=0, sample=None, lite=False, muon=False):
+             pad=0, sample=None, lite=False, muon=False, combined=False):
     """shapes: list of (batch, rows, cols).  `pad` adds that many elements between stacked matrices
     (batch_stride > rows*cols).  `sample`: dict spec index -> list of batch indices the oracle follows
     (default: all).  Returns dict of max relative errors over steps and sampled matrices."""
@@ -84,7 +84,7 @@ def run_case(shapes, steps=3, hp=None, grad_dtype=torch.float32, rho=0.9, sigma=
     gbufs, gviews = zip(*[device_buffer(g, grad_dtype) for g in grads_seq[0]])
     obufs, oviews = zip(*[device_buffer(torch.zeros_like(w), torch.float32) for w in W0])
 
-    descs = [pkg.MatrixDesc(s[1], s[2], s[0], s[1] * s[2] + pad, 1 if grad_dtype == torch.bfloat16 else 0, 1 if lite else 0) for s in shapes]
+    descs = [pkg.MatrixDesc(s[1], s[2], s[0], s[1] * s[2] + pad, 1 if grad_dtype == torch.bfloat16 else 0, 2 if combined else (1 if lite else 0)) for s in shapes]
     opt = pkg.MonaOptimizer.__new__(pkg.MonaOptimizer)
     _init_from_descs(opt, descs, dev)
 
@@ -107,6 +107,18 @@ def run_case(shapes, steps=3, hp=None, grad_dtype=torch.float32, rho=0.9, sigma=
                 Wn, O = step_fn(Wref[(i, b)], grads_seq[k][i][b].double().numpy(), states[(i, b)], ohp)
                 Wref[(i, b)] = Wn
                 s = states[(i, b)]
+                if combined:
+                    # the library keeps Z_k = beta_a A_k - (1 - beta_a) G_k; the same combination of the oracle's state
+                    z_ref = ohp.accel_beta * s.A - (1.0 - ohp.accel_beta) * s.G_prev
+                    errs["M"] = max(errs["M"], rel(Mv[b].cpu().numpy(), s.M))
+                    errs["A"] = max(errs["A"], rel(Av[b].double().cpu().numpy(), z_ref))
+                    assert Gv is None
+                    errs["O"] = max(errs["O"], rel(oviews[i][b].cpu().numpy(), O))
+                    got = pviews[i][b].double().cpu().numpy()
+                    w0 = W0[i][b].double().numpy()
+                    errs["W"] = max(errs["W"], rel(got, Wn))
+                    errs["dW"] = max(errs["dW"], rel(got - w0, Wn - w0))
+                    continue
                 a_gpu, g_gpu = Av[b].double().cpu().numpy(), Gv[b].double().cpu().numpy()
                 errs["M"] = max(errs["M"], rel(Mv[b].cpu().numpy(), s.M))
                 errs["A"] = max(errs["A"], rel(a_gpu, s.A))

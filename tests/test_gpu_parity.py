@@ -108,6 +108,17 @@ def test_paper_expert_shapes(shape):
     check(errs, TOL_O_BF16)
 
 
+@pytest.mark.parametrize("shapes,grad_dtype,steps", [([(1, 256, 512)], torch.float32, 5), ([(2, 512, 256), (1, 32, 1024), (1, 33, 17)], torch.float32, 10),
+                                                     ([(3, 128, 384)], torch.bfloat16, 4)])
+def test_single_buffer_state_format(shapes, grad_dtype, steps):
+    """state_dtype = MONA_STATE_COMBINED: one fp32 buffer Z_k = beta_a A_k - (1 - beta_a) G_k instead of A_k and
+    G_{k-1}.  Same step as Algorithm 1: M, O and W against the oracle as usual, Z against the same combination
+    of the oracle's A_k and G_k, all to the fp32 state tolerance."""
+    errs = run_case(shapes, steps=steps, grad_dtype=grad_dtype, seed=23, combined=True)
+    assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE, errs
+    assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
+
+
 def test_plain_muon_path():
     """algorithm = 1: Eq. muon_momentum without the acceleration term; A and G_prev are neither read nor written
     (they stay at their initial zero, so their error against the oracle's untouched zero state is exactly 0)."""

@@ -47,6 +47,8 @@ def test_query_sizes_state_is_three_fp32_per_parameter(L):
     lite = [pkg.MatrixDesc(x.rows, x.cols, x.batch, 0, 0, 1) for x in d]
     sb_lite, _ = pkg.query_sizes(lite)
     assert 8 * n <= sb_lite <= 8 * n + 9 * 256      # bfloat16 storage of A and G_prev: 4 + 2 + 2 bytes per parameter
+    single = [pkg.MatrixDesc(x.rows, x.cols, x.batch, 0, 0, pkg.MONA_STATE_COMBINED) for x in d]
+    assert 8 * n <= pkg.query_sizes(single)[0] <= 8 * n + 6 * 256   # M and the single buffer Z
     assert wb > 0
     # same shapes share one bucket: once the chunk is bounded by the budget (not by the matrix count),
     # two descriptors of one shape need the workspace of one
