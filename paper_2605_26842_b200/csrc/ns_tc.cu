@@ -447,6 +447,60 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                 const uint32_t acc = acc0 + u;
                 const int n0 = (tc.tn + u) * TC_BN;
                 const int nphases = (g.N - n0 > EPI_COLS) ? 2 : 1;
+                if constexpr (WIDE) {
+                    // Macro-tile configuration (no axpy operand, no diagonal term): both accumulators belong to the tile
+                    // in flight, so nothing hides this epilogue.  A thread's share of an accumulator (128 values) fits
+                    // in 64 packed registers: read and pack all of it first, hand the accumulator back to the MMA issuer,
+                    // and only then stage and store.
+                    bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
+                    ok = epi_bar_all(3, ok);
+                    if (!ok) { alive = false; break; }
+                    tc_fence_after();
+                    acc_par ^= 1u << acc;
+                    const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
+                    uint4 pk[2][8];
+                    #pragma unroll
+                    for (int ph = 0; ph < 2; ++ph) {
+                        if (ph < nphases) {
+                            float v[64];
+                            tmem_ld32(t_base + ph * EPI_COLS, v);
+                            tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
+                            tmem_ld_wait();
+                            #pragma unroll
+                            for (int j = 0; j < 64; ++j) v[j] *= c2;
+                            #pragma unroll
+                            for (int q = 0; q < 8; ++q) pk[ph][q] = pack8(v + 8 * q);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8 * acc);
+                    #pragma unroll
+                    for (int ph = 0; ph < 2; ++ph) {
+                        if (ph < nphases) {
+                            const uint32_t buf = epi_base + (epi_it % C::EPI_BUFS) * EPI_BUF_BYTES;
+                            if (issuer) bulk_wait_read<C::EPI_BUFS - 1>();
+                            epi_bar_sync(1);
+                            #pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const uint32_t addr = buf + stage_off + (((uint32_t)q ^ swz) << 4);
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[ph][q].x), "r"(pk[ph][q].y),
+                                             "r"(pk[ph][q].z), "r"(pk[ph][q].w) : "memory");
+                            }
+                            fence_proxy_async();
+                            epi_bar_sync(2);
+                            if (issuer) {
+                                #pragma unroll
+                                for (int b = 0; b < 4; ++b) {
+                                    const int x = n0 + ph * EPI_COLS + (b & 1) * TC_BOX, y = m0 + (b >> 1) * TC_BOX;
+                                    if (x < g.N && y < g.M) tma_store_3d(&tma_d, buf + b * BOX_BYTES, x, y, tc.c);
+                                }
+                                bulk_commit();
+                            }
+                            ++epi_it;
+                        }
+                    }
+                } else {
                 // operand of the axpy term, requested before the accumulator is ready
                 uint4 cin_raw[8];
                 auto load_cin = [&](int ph) {
@@ -520,7 +574,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                     }
                     ++epi_it;
                 }
-            }
+                            }
+}
             if (!WIDE) acc_next ^= 1u;
         }
         if (issuer) bulk_wait_all();           // shared memory must outlive the stores that read it
