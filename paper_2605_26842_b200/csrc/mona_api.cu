@@ -41,8 +41,6 @@ static_assert(sizeof(unsigned int) * MAXC <= CTRL_INVNORM_OFF && sizeof(float) *
 
 // 1: consecutive chunks are pipelined over two streams; 0: everything runs on the caller's stream.
 int g_chunk_overlap = 1;
-// 1: X' = B' X runs on 256 x 512 macro-tiles.
-int g_wide_g3 = 1;
 
 // Bytes of bf16 iterates (X_t, X_{t+1}, A_t, B_t) a chunk may hold so that it stays resident in L2
 // between the 3T GEMMs of the iteration.
@@ -68,7 +66,7 @@ struct Bucket {
     size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;          // bf16 mode, bytes from the slot's iterate base
     size_t off32_x[2] = {0, 0}, off32_a = 0, off32_b = 0;    // fp32 mode
     size_t data_bytes = 0;
-    CUtensorMap tm_x[NSLOTS][2], tm_a[NSLOTS], tm_b[NSLOTS];
+    CUtensorMap tm_x[NSLOTS][2] = {}, tm_a[NSLOTS] = {}, tm_b[NSLOTS] = {};
 };
 
 struct Plan {
@@ -179,7 +177,7 @@ F2 split(double v) {
 
 struct mona_handle {
     Plan plan;
-    int device = 0, num_sms = 0, max_pairs = 0;
+    int device = 0, max_pairs = 0;
     uint8_t* state = nullptr;
     uint8_t* ws = nullptr;
     cudaStream_t side = nullptr;
@@ -264,7 +262,6 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
     MONA_CUDA(h, cudaGetDeviceProperties(&prop, device));
     if (prop.major != 10) return h->fail(MONA_ERR_ARCH, "device %d is sm_%d%d; this library is built for sm_100a only", device, prop.major, prop.minor);
     h->device = device;
-    h->num_sms = prop.multiProcessorCount;
     h->state = (uint8_t*)state;
     h->ws = (uint8_t*)workspace;
 
@@ -420,7 +417,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                         tc_gemm_plan(g2);
                         MONA_CUDA(h, launch_tc_gemm(b.tm_a[slot], b.tm_a[slot], b.tm_b[slot], g2, h->max_pairs, dstatus, stream));
                         TcGemm g3{};
-                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0; g3.wide = g_wide_g3;
+                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0; g3.wide = 1;   // 256 x 512 macro-tiles
                         g3.cin = nullptr; g3.c1 = 0.f; g3.c2 = 1.f;
                         g3.inv_norm = inv_norm; g3.post_mode = t == 0 ? 1 : 0;
                         if (!b.tall) {   // X' = B' X : B' is the symmetric "A" operand, X the MN-major "B" operand
