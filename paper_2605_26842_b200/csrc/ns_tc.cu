@@ -18,8 +18,9 @@
 // products, here X' = B' X) a pair computes a 256 x 512 macro-tile, i.e. two neighbouring tiles at once,
 // one per accumulator, from ONE staged slice of the A operand: 96 KiB instead of 128 KiB cross from L2
 // per k-slice and pair.  The main loop is bound by that traffic, not by the tensor pipe, so fewer bytes
-// per flop is worth more than accumulator double-buffering; the operand ring keeps filling while the
-// epilogue drains, which hides most of it.
+// per flop is worth more than accumulator double-buffering.  To keep the unhidden part of that epilogue short,
+// its warps first read and pack a whole accumulator into registers and hand it back to the MMA issuer, and only
+// then stage and store; the operand ring keeps filling meanwhile.
 //
 // Every wait on an mbarrier is bounded: when one runs out the CTA latches STATUS_TIMEOUT, raises its
 // abort flag, and all roles fall through to the common exit, where tensor memory is released.
@@ -38,7 +39,7 @@ namespace {
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
 constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
-// 320 threads x 160 registers leave room on the SM for one 256-thread block of the elementwise kernels
+// 320 threads x 160 registers: no spills, and room is left on the SM for one 256-thread block of another kernel
 constexpr int TC_MAX_REGS = 160;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
