@@ -27,3 +27,13 @@ def test_one_layer_of_the_7b_set_sampled():
     # buckets: 128 wide experts (2 chunks), 64 tall experts, 4 attention matrices, 1 shared expert: 5 chunks,
     # each one prologue + 15 GEMMs + one update
     assert errs["launches"] == 5 * 17, errs["launches"]
+
+
+def test_shard_stress_shapes_with_bf16_gradients():
+    """The shapes of the large-MoE shard configuration (1024x4096 experts wide and tall, 4096x4096 attention),
+    bfloat16 gradients, its beta_a = 0.975 / alpha = -20: two steps, every matrix followed by the oracle."""
+    import torch
+    hp = pkg.default_hparams(accel_beta=0.975, accel_alpha=-20.0)
+    errs = run_case([(2, 1024, 4096), (1, 4096, 1024), (1, 4096, 4096)], steps=2, hp=hp, grad_dtype=torch.bfloat16, seed=1238)
+    assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE and errs["Gprev"] <= TOL_STATE, errs
+    assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
