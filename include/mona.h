@@ -166,6 +166,14 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp,
  * reported a problem, or -1.  The word is cleared by the call. */
 mona_status mona_poll_status(mona_handle* h, void* stream, int64_t* first_bad_matrix);
 
+/* Failure-detection self-test: enqueues one Newton-Schulz GEMM launch whose shared-memory stages are made to
+ * expect 16 bytes more than their copies deliver.  Nothing faults - every copy completes - but the wait for a
+ * full stage can never end, so it must run out after its bound (about half a second), latch the time-out in the
+ * status word and leave the kernel cleanly.  Afterwards mona_poll_status() returns MONA_ERR_TIMEOUT once and
+ * the handle works as before.  Only the first workspace slot is written (with meaningless values); parameters
+ * and state are not touched.  Needs at least one descriptor that takes the tensor-core path. */
+mona_status mona_selftest_timeout(mona_handle* h, void* stream);
+
 /* Byte offsets inside the state block of M, A and G_prev of matrix 0 of descriptor `desc`.  Matrix b
  * of the descriptor follows at b * rows * cols * (element size) bytes from each offset: 4 for M, and 4
  * or 2 for A and G_prev according to the descriptor's state_dtype (state is stored densely, whatever

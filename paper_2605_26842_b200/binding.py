@@ -57,6 +57,8 @@ def lib() -> C.CDLL:
     L.mona_step_ex.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, C.c_uint32, vp]
     L.mona_step_host.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, vpp, vp]
     L.mona_poll_status.argtypes = [vp, vp, C.POINTER(C.c_int64)]
+    L.mona_selftest_timeout.argtypes = [vp, vp]
+    L.mona_selftest_timeout.restype = C.c_int
     L.mona_state_layout.argtypes = [vp, C.c_int64, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.mona_last_launch_count.argtypes = [vp]
     L.mona_last_launch_count.restype = C.c_int64
@@ -178,6 +180,10 @@ class MonaOptimizer:
         bad = C.c_int64(-1)
         st = lib().mona_poll_status(self._h, self._stream(), C.byref(bad))
         return st, bad.value
+
+    def selftest_timeout(self):
+        """Enqueues the launch whose wait must run out; poll_status() then reports MONA_ERR_TIMEOUT once."""
+        self._check(lib().mona_selftest_timeout(self._h, self._stream()))
 
     def state_layout(self, desc: int):
         a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()

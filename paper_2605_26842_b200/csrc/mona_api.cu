@@ -563,6 +563,23 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp, void* const* 
     return MONA_OK;
 }
 
+mona_status mona_selftest_timeout(mona_handle* h, void* stream_v) {
+    if (!h) return MONA_ERR_INVALID_ARG;
+    MONA_CUDA(h, cudaSetDevice(h->device));
+    for (const Bucket& b : h->plan.buckets) {
+        if (!b.tc_ok) continue;
+        // one X X^T launch over the first matrix slot of the workspace whose stages expect 16 bytes too many
+        TcGemm g{};
+        g.C = 1; g.M = g.N = (int)b.s; g.K = (int)b.l; g.a_mn = g.b_mn = b.tall ? 1 : 0; g.symmetric = 1; g.ab_same = 1;
+        g.c1 = 0.f; g.c2 = 1.f; g.inv_norm = (const float*)(h->ws + WS_CTRL_OFF + CTRL_INVNORM_OFF); g.post_mode = 0;
+        g.selftest_extra_tx = 16;
+        tc_gemm_plan(g);
+        MONA_CUDA(h, launch_tc_gemm(b.tm_x[0][0], b.tm_x[0][0], b.tm_a[0], g, h->max_pairs, (DeviceStatus*)(h->ws + WS_STATUS_OFF), (cudaStream_t)stream_v));
+        return MONA_OK;
+    }
+    return h->fail(MONA_ERR_UNSUPPORTED_SHAPE, "no descriptor of this handle takes the tensor-core path");
+}
+
 mona_status mona_poll_status(mona_handle* h, void* stream_v, int64_t* first_bad_matrix) {
     if (!h) return MONA_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)stream_v;

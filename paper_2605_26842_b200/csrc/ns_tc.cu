@@ -336,7 +336,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                 const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand (first sub-tile)
                 // diagonal tile of X X^T or A A: both operands are the same rows, staged once
                 const bool shared_ab = !WIDE && g.ab_same && tc.tm == tc.tn;
-                const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (shared_ab ? 0u : (uint32_t)tc.nsub * B_SUB_BYTES));
+                const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (shared_ab ? 0u : (uint32_t)tc.nsub * B_SUB_BYTES)) + (uint32_t)g.selftest_extra_tx;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1))) break;
                     const uint32_t full = full_leader + 8 * stage;

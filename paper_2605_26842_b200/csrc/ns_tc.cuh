@@ -39,6 +39,9 @@ struct TcGemm {
     float diag_add;             // added to D(i,i): folds the a*X term of the quintic into B' = b A + c A^2 + a I
     const float* inv_norm;      // per-matrix 1/(||M||_F + eps), used when post_mode != 0
     int post_mode;              // 0: post = 1, 1: post = inv, 2: post = inv^2
+    int selftest_extra_tx;      // 0 in normal use.  The time-out self-test sets it: every stage then expects this many
+                                //    bytes more than its copies deliver, so the "full" wait runs out and the kernel must
+                                //    report STATUS_TIMEOUT and leave cleanly (all copies still complete; nothing faults)
 };
 
 // Fills the tile counts of `g` from M, N, symmetric, wide.

@@ -257,3 +257,25 @@ def test_chunk_overlap_does_not_change_results():
     finally:
         pkg.set_chunk_overlap(True)
         pkg.set_chunk_budget(768 << 20)
+
+
+def test_a_wait_that_cannot_end_times_out_and_the_handle_survives():
+    """Failure detection without a fault: a launch whose stages expect bytes that never come must give up after its
+    bounded wait, report MONA_ERR_TIMEOUT through the status word, release tensor memory and leave the context
+    usable - the next step on the same handle is correct."""
+    import time
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(3)
+    p = [(torch.randn(1, 256, 512, generator=gen) * 0.02).to(dev)]
+    g = [(torch.randn(1, 256, 512, generator=gen) * 1e-3).to(dev)]
+    opt = pkg.MonaOptimizer(p)
+    t0 = time.time()
+    opt.selftest_timeout()
+    st, bad = opt.poll_status()
+    assert pkg.STATUS_NAMES[st] == "MONA_ERR_TIMEOUT", (st, bad)
+    assert time.time() - t0 < 20.0
+    assert opt.poll_status()[0] == 0                 # latched once, then cleared
+    opt.close()
+    # same device, fresh handle and a full parity case: nothing was left behind
+    errs = run_case([(1, 256, 512)], steps=2, seed=5)
+    check(errs, TOL_O_BF16)
