@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised in profiles/tc_gemm_kernel_moe7b_768x2048_per_launch.md: mean over the 15 launches of one 93-matrix
 # 768x2048 chunk, the launch shape that makes up most of the default workload.  Valid only for the kernel source
 # the counters were taken with (hash of ns_tc.cu + ns_tc.cuh).
-NCU_TRAFFIC = {"source_sha256_16": "3ee10f64ac07c4a8", "bytes_per_launch": 358.5e6}
+NCU_TRAFFIC = {"source_sha256_16": "553d71a096c0df77", "bytes_per_launch": 357.1e6}
 
 
 def kernel_traffic():
