@@ -322,6 +322,17 @@ def main():
     # ---- end to end: host gradients in, host parameters out, through mona_step_host ----
     e2e = None
     if not args.no_e2e:
+        # the pinned host copies of all gradients and parameters must fit the node for every rank at once
+        need = sum(g.numel() * g.element_size() for g in gp.grads) + sum(p.numel() * p.element_size() for p in params)
+        try:
+            import psutil
+            avail = psutil.virtual_memory().available
+        except Exception:
+            avail = None
+        if avail is not None and need * world > 0.6 * avail:
+            e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                   "error": f"skipped: {world} rank(s) x {need / 1e9:.1f} GB of pinned host memory against {avail / 1e9:.1f} GB available"}
+    if not args.no_e2e and e2e is None:
         try:
             g_host = [torch.empty(g.shape, dtype=g.dtype, pin_memory=True) for g in gp.grads]
             p_host = [torch.empty(p.shape, dtype=p.dtype, pin_memory=True) for p in params]
