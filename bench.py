@@ -329,6 +329,8 @@ def main():
             avail = psutil.virtual_memory().available
         except Exception:
             avail = None
+        if dist is not None:    # every rank must take the same branch: use the smallest figure any rank saw
+            avail = -shard.max_over_ranks(-float(avail if avail is not None else 0.0), dist, dev)
         if avail is not None and need * world > 0.6 * avail:
             e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                    "error": f"skipped: {world} rank(s) x {need / 1e9:.1f} GB of pinned host memory against {avail / 1e9:.1f} GB available"}
