@@ -24,6 +24,9 @@
  *     small host/device tables, one internal stream and a few events.
  *   - Every function returns a mona_status; nothing throws or aborts.  Problems detected on the device
  *     (non-finite norm, a wait that ran out) are latched in a status word read by mona_poll_status().
+ *     A step that reported MONA_ERR_TIMEOUT or MONA_ERR_NONFINITE has already advanced M, A and G_prev and
+ *     may have written parameters from incomplete iterates: restore state and parameters from the caller's
+ *     last checkpoint before stepping again.
  *   - There is no CPU fallback: on a machine without an sm_100 device mona_create() fails with
  *     MONA_ERR_ARCH / MONA_ERR_CUDA.
  *   - One handle is used from one host thread and one stream at a time.
@@ -106,22 +109,51 @@ typedef struct mona_handle mona_handle;
  * eps = 1e-7 where it does not. */
 mona_status mona_default_hparams(mona_hparams* hp);
 
-/* Tuning knob, process-wide: bytes of bf16 Newton-Schulz iterates (X_t, X_{t+1}, A_t, B_t) one chunk of
- * same-shape matrices may hold.  A chunk goes through all 3T GEMMs of the iteration before the next one
- * starts, so it should fit the L2 cache.  Default 48 MiB; at least 1 MiB.  Affects later calls of
- * mona_query_sizes() and mona_create() only. */
-mona_status mona_set_chunk_budget(size_t bytes);
+/* Per-handle tuning options.  Obtain the defaults with mona_default_options(), change what you need, and pass
+ * the SAME struct to mona_query_sizes_opt() and mona_create_opt(): the workspace size depends on it.  A handle
+ * keeps the options it was created with.
+ *   chunk_budget_bytes : bytes of bf16 Newton-Schulz iterates (X_t, X_{t+1}, A_t, B'_t) one chunk of same-shape
+ *                        matrices may hold (0 = the default, 768 MiB; otherwise at least 1 MiB).  A chunk goes
+ *                        through prologue, the whole iteration and the update before the next one starts.
+ *                        Chunks are sized to keep every SM pair busy, not to fit a cache: cache-sized chunks
+ *                        (tens of MiB) hold too few tiles for the machine and were measured 1.5-2x slower.
+ *   chunk_overlap      : 1 (default) pipelines consecutive chunks over two streams - the caller's and one the
+ *                        handle owns, joined by events before mona_step*() returns to the caller's stream - so
+ *                        that the start and the tail of one chunk's kernels are filled by the other chunk's;
+ *                        0 keeps every launch on the caller's stream.  Results are identical either way; the
+ *                        workspace holds two chunks.
+ *   fuse_update        : 1 (default): on the tensor-core path the last X' = B' X of a step applies Eq. muon_update
+ *                        in its epilogue (fp32 O_k straight from the accumulator, no bf16 copy of O_k written and
+ *                        re-read, no separate update kernel).  0: O_k is stored in bf16 and a separate elementwise
+ *                        kernel updates the parameters.  The two differ by the bf16 rounding of O_k only.
+ *   ns_delay           : how many matrices apart consecutive Newton-Schulz GEMMs of one matrix sit in the kernel's
+ *                        work order (0 = the default, 3; at most 64).  Larger values hide the dependency latency
+ *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it. */
+typedef struct {
+    size_t chunk_budget_bytes;
+    int32_t chunk_overlap;
+    int32_t fuse_update;
+    int32_t ns_delay;
+    int32_t reserved[5];       /* zero */
+} mona_options;
 
-/* Tuning knob, process-wide: 1 (default) pipelines consecutive chunks over two streams - the caller's and
- * one the handle owns, joined by events before mona_step*() returns to the caller's stream - so that the
- * partial last wave and the launch gap of one chunk's kernels are filled by the other chunk's; 0 keeps
- * every launch on the caller's stream.  Results are identical either way; the workspace holds two chunks. */
+/* Fills *opt with the defaults (as changed by the two process-wide setters below, if they were called). */
+mona_status mona_default_options(mona_options* opt);
+
+/* Process-wide defaults that seed mona_default_options() and the plain mona_query_sizes()/mona_create():
+ * chunk budget in bytes (at least 1 MiB) and chunk overlap (0/1).  They affect handles created later only; an
+ * existing handle keeps its own options.  Prefer the options struct: these two exist for callers that create
+ * all their handles with one setting, and must not be changed between mona_query_sizes() and mona_create(). */
+mona_status mona_set_chunk_budget(size_t bytes);
 mona_status mona_set_chunk_overlap(int enabled);
 
 /* Bytes the caller must provide for the optimizer state (M, A, G_prev, Algorithm 1 line 1: 12 bytes per
  * parameter, 8 with bfloat16 storage of A and G_prev) and for the Newton-Schulz workspace.  Host only; no device is touched. */
 mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc,
                              size_t* state_bytes, size_t* workspace_bytes);
+/* The same with explicit options (NULL = defaults). */
+mona_status mona_query_sizes_opt(const mona_matrix_desc* descs, int64_t n_desc, const mona_options* options,
+                                 size_t* state_bytes, size_t* workspace_bytes);
 
 /* Builds the plan (shape buckets, chunking, tile schedules, TMA descriptors) for `n_desc` descriptors
  * on CUDA device `device`, binds the caller's state and workspace blocks (both 256-byte aligned device
@@ -130,6 +162,10 @@ mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc,
 mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc,
                         void* state, size_t state_bytes, void* workspace, size_t workspace_bytes,
                         int device);
+/* The same with explicit options (NULL = defaults); sizes must come from mona_query_sizes_opt() with the same options. */
+mona_status mona_create_opt(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc,
+                            const mona_options* options, void* state, size_t state_bytes, void* workspace,
+                            size_t workspace_bytes, int device);
 
 /* One optimizer step for all descriptors, enqueued on `stream` (a cudaStream_t passed as void*;
  * NULL = the legacy default stream).  params[i] / grads[i] are the device base pointers of
@@ -166,7 +202,7 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp,
  * reported a problem, or -1.  The word is cleared by the call. */
 mona_status mona_poll_status(mona_handle* h, void* stream, int64_t* first_bad_matrix);
 
-/* Failure-detection self-test: enqueues one Newton-Schulz GEMM launch whose shared-memory stages are made to
+/* Failure-detection self-test: enqueues one Newton-Schulz launch (a single X X^T phase) whose shared-memory stages are made to
  * expect 16 bytes more than their copies deliver.  Nothing faults - every copy completes - but the wait for a
  * full stage can never end, so it must run out after its bound (about half a second), latch the time-out in the
  * status word and leave the kernel cleanly.  Afterwards mona_poll_status() returns MONA_ERR_TIMEOUT once and
@@ -185,9 +221,12 @@ mona_status mona_state_layout(const mona_handle* h, int64_t desc,
 int64_t mona_last_launch_count(const mona_handle* h);
 
 /* Counts of executed tensor-core work of the most recent step: bf16 multiply-add flops actually
- * issued (2 * M * N * K summed over issued tile MMAs) and the dense-equivalent figure
- * (4 s^2 l + 2 s^3 per matrix and iteration).  Either pointer may be NULL. */
+ * issued (2 * M * N * K summed over issued 256 x 256 tile MMAs: padding and the upper halves of diagonal tiles
+ * count) and the dense-equivalent figure (4 s^2 l + 2 s^3 per matrix and iteration).  Either pointer may be NULL. */
 mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* dense_equivalent);
+/* The work the iteration itself needs when both symmetric products are computed once per pair of entries:
+ * 3 s^2 l + s^3 per matrix and iteration (tensor-core path only). */
+mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful);
 
 /* Allocation-free prologue for ONE matrix.  The paper has no counterpart to this entry point; it exists
  * for integration reasons only.  It performs lines 4-7 and 10 of Algorithm 1 on a rows x cols matrix
@@ -209,6 +248,11 @@ mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* d
  *   - All calls on a device share the one array, and it keeps the previous call's contents (the function
  *     re-zeroes the counter it depends on).  Two calls whose kernels may overlap on the GPU - different
  *     streams, no ordering between them - race on it; order them yourself.
+ *   - hp->algorithm must be 0 (the plain-Muon prologue has no acceleration state to update).
+ *   - There is no status word to poll here.  A gradient or state holding inf/nan shows in the result itself:
+ *     a finite ||M_k||_F always gives a positive finite inv_norm_out[0]; a non-finite one gives 0 (norm = inf)
+ *     or nan.  Test inv_norm_out[0] before using M_k.
+ *   - A device that is not compute capability 10.x is refused with MONA_ERR_ARCH.
  *   - `err` (may be NULL) receives a NUL-terminated message of at most err_len bytes.
  * Enqueued on `stream`; does not synchronise. */
 mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtype, float* M, float* A, float* G_prev,

@@ -35,6 +35,12 @@ class Hparams(C.Structure):
                 ("ns_precision", C.c_int32), ("algorithm", C.c_int32)]
 
 
+class Options(C.Structure):
+    """mona_options: per-handle tuning knobs (see include/mona.h)."""
+    _fields_ = [("chunk_budget_bytes", C.c_size_t), ("chunk_overlap", C.c_int32), ("fuse_update", C.c_int32),
+                ("ns_delay", C.c_int32), ("reserved", C.c_int32 * 5)]
+
+
 _lib = None
 
 
@@ -52,6 +58,10 @@ def lib() -> C.CDLL:
     L.mona_set_chunk_budget.argtypes = [C.c_size_t]
     L.mona_set_chunk_overlap.argtypes = [C.c_int]
     L.mona_query_sizes.argtypes = [C.POINTER(MatrixDesc), C.c_int64, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.mona_default_options.argtypes = [C.POINTER(Options)]
+    L.mona_query_sizes_opt.argtypes = [C.POINTER(MatrixDesc), C.c_int64, C.POINTER(Options), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+    L.mona_create_opt.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, C.POINTER(Options), vp, C.c_size_t, vp, C.c_size_t, C.c_int]
+    L.mona_last_ns_useful_flops.argtypes = [vp, C.POINTER(C.c_double)]
     L.mona_create.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_step.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vp]
     L.mona_step_ex.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, C.c_uint32, vp]
@@ -68,7 +78,8 @@ def lib() -> C.CDLL:
     L.mona_destroy.argtypes = [vp]
     L.mona_destroy.restype = None
     for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_set_chunk_overlap", "mona_query_sizes", "mona_create", "mona_step",
-                 "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops"):
+                 "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops",
+                 "mona_default_options", "mona_query_sizes_opt", "mona_create_opt", "mona_last_ns_useful_flops"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -84,6 +95,18 @@ def default_hparams(**overrides) -> Hparams:
             raise AttributeError(k)
         setattr(hp, k, v)
     return hp
+
+
+def default_options(**overrides) -> Options:
+    opt = Options()
+    st = lib().mona_default_options(C.byref(opt))
+    if st:
+        raise MonaError(st)
+    for k, v in overrides.items():
+        if not hasattr(opt, k):
+            raise AttributeError(k)
+        setattr(opt, k, v)
+    return opt
 
 
 def set_chunk_budget(nbytes: int) -> None:
@@ -105,9 +128,10 @@ def _desc_array(descs: Sequence[MatrixDesc]):
     return arr
 
 
-def query_sizes(descs: Sequence[MatrixDesc]):
+def query_sizes(descs: Sequence[MatrixDesc], options: Optional[Options] = None):
     sb, wb = C.c_size_t(0), C.c_size_t(0)
-    st = lib().mona_query_sizes(_desc_array(descs), len(descs), C.byref(sb), C.byref(wb))
+    st = lib().mona_query_sizes_opt(_desc_array(descs), len(descs), None if options is None else C.byref(options),
+                                    C.byref(sb), C.byref(wb))
     if st:
         raise MonaError(st, "mona_query_sizes")
     return sb.value, wb.value
@@ -128,7 +152,7 @@ class MonaOptimizer:
     torch stream."""
 
     def __init__(self, params: Sequence[torch.Tensor], grad_dtype=torch.float32, device: Optional[int] = None,
-                 state_dtype=torch.float32):
+                 state_dtype=torch.float32, options: Optional[Options] = None):
         L = lib()
         self.descs: List[MatrixDesc] = []
         for p in params:
@@ -141,13 +165,14 @@ class MonaOptimizer:
                                          (MONA_BF16 if state_dtype == torch.bfloat16 else MONA_F32)))
         self.device = torch.cuda.current_device() if device is None else device
         self.grad_dtype = grad_dtype
-        sb, wb = query_sizes(self.descs)
+        self.options = options if options is not None else default_options()
+        sb, wb = query_sizes(self.descs, self.options)
         dev = torch.device("cuda", self.device)
         self.state = torch.empty(sb, dtype=torch.uint8, device=dev)
         self.workspace = torch.empty(wb, dtype=torch.uint8, device=dev)
         self._h = C.c_void_p()
-        st = L.mona_create(C.byref(self._h), _desc_array(self.descs), len(self.descs), self.state.data_ptr(), sb,
-                           self.workspace.data_ptr(), wb, self.device)
+        st = L.mona_create_opt(C.byref(self._h), _desc_array(self.descs), len(self.descs), C.byref(self.options),
+                               self.state.data_ptr(), sb, self.workspace.data_ptr(), wb, self.device)
         if st:
             msg = L.mona_last_error(self._h).decode() if self._h else ""
             L.mona_destroy(self._h)
@@ -214,6 +239,11 @@ class MonaOptimizer:
         e, d = C.c_double(), C.c_double()
         self._check(lib().mona_last_ns_flops(self._h, C.byref(e), C.byref(d)))
         return e.value, d.value
+
+    def last_ns_useful_flops(self) -> float:
+        u = C.c_double()
+        self._check(lib().mona_last_ns_useful_flops(self._h, C.byref(u)))
+        return u.value
 
     def close(self):
         if getattr(self, "_h", None):

@@ -8,11 +8,20 @@
 namespace mona {
 
 // A chunk is the unit that goes through prologue -> Newton-Schulz -> update together: up to MAXC
-// same-shape matrices whose bf16 iterates fit the L2 budget.
+// same-shape matrices whose bf16 iterates fit the chunk budget (sized for full machine occupancy, not for cache).
 constexpr int MAXC = 512;   // the pointer table below travels as a kernel argument (14 KiB of the 32 KiB CUDA 12 allows)
 // Each matrix is cut into at most MAX_SLABS contiguous slabs for the elementwise passes; every slab
 // owns one partial sum of squares, so the Frobenius norm is reduced in a fixed order.
 constexpr int MAX_SLABS = 256;
+
+// Slab decomposition of a matrix of e elements: ~16 K elements per slab, at most MAX_SLABS slabs, slab length a
+// multiple of 1024 once the cap binds.
+inline void slab_plan(long long e, long long* slab_len, int* slabs) {
+    long long slab = 16384;
+    if ((e + slab - 1) / slab > MAX_SLABS) slab = ((e + MAX_SLABS - 1) / MAX_SLABS + 1023) / 1024 * 1024;
+    *slab_len = slab;
+    *slabs = (int)((e + slab - 1) / slab);
+}
 
 // Per-chunk pointer table passed by value to the elementwise kernels.
 struct ChunkPtrs {

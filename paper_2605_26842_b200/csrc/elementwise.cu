@@ -363,7 +363,7 @@ struct NoAllocScratch {
     float partials[MAX_SLABS];     // slab sums of squares (fully rewritten by every call)
     unsigned int counter;          // slab arrival counter; must be 0 when a call starts
     unsigned int pad[3];
-    DeviceStatus status;           // non-finite flag sink (not reported by this entry point)
+    DeviceStatus status;           // sink of the kernel's non-finite flag; the caller reads inv_norm_out instead
 };
 static_assert(sizeof(NoAllocScratch) <= 2048, "scratch layout");
 
@@ -372,6 +372,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[2048];
 
 std::mutex g_noalloc_mutex;
 NoAllocScratch* g_noalloc_dev_ptr[NOALLOC_MAX_DEVICES] = {nullptr};
+int g_noalloc_dev_major[NOALLOC_MAX_DEVICES] = {0};
 
 void set_msg(char* buf, size_t len, const char* msg) {
     if (buf && len) {
@@ -398,6 +399,7 @@ extern "C" mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtyp
     if (!grad || !M || !A || !G_prev || !inv_norm_out || !hp) { set_msg(err, err_len, "null pointer argument"); return MONA_ERR_INVALID_ARG; }
     if (rows <= 0 || cols <= 0) { set_msg(err, err_len, "rows and cols must be positive"); return MONA_ERR_INVALID_ARG; }
     if (grad_dtype != MONA_F32 && grad_dtype != MONA_BF16) { set_msg(err, err_len, "unknown grad_dtype"); return MONA_ERR_INVALID_ARG; }
+    if (hp->algorithm != 0) { set_msg(err, err_len, "this entry point runs the MONA prologue only (hp->algorithm must be 0)"); return MONA_ERR_INVALID_ARG; }
     if (rows > NOALLOC_MAX_ELEMS || cols > NOALLOC_MAX_ELEMS || rows * cols > NOALLOC_MAX_ELEMS) {
         set_msg(err, err_len, "matrix larger than the built-in scratch supports: rows*cols must be <= 16777216 (4096 x 4096)");
         return MONA_ERR_UNSUPPORTED_SHAPE;
@@ -417,15 +419,20 @@ extern "C" mona_status mona_prologue_noalloc(const void* grad, int32_t grad_dtyp
             void* p = nullptr;
             ce = cudaGetSymbolAddress(&p, g_noalloc_scratch);
             if (ce != cudaSuccess || !p) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
+            int major = 0;
+            ce = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+            if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }
+            g_noalloc_dev_major[dev] = major;
             g_noalloc_dev_ptr[dev] = reinterpret_cast<NoAllocScratch*>(p);
         }
+        if (g_noalloc_dev_major[dev] != 10) { set_msg(err, err_len, "the current device is not compute capability 10.x"); return MONA_ERR_ARCH; }
         scratch = g_noalloc_dev_ptr[dev];
     }
     cudaStream_t stream = (cudaStream_t)stream_v;
     const long long e = rows * cols;
-    long long slab = 16384;
-    if ((e + slab - 1) / slab > MAX_SLABS) slab = ((e + MAX_SLABS - 1) / MAX_SLABS + 1023) / 1024 * 1024;
-    const int slabs = (int)((e + slab - 1) / slab);
+    long long slab = 0;
+    int slabs = 0;
+    slab_plan(e, &slab, &slabs);
     // the array keeps whatever the previous call left: the counter has to start from zero
     ce = cudaMemsetAsync(&scratch->counter, 0, sizeof(unsigned int), stream);
     if (ce != cudaSuccess) { set_msg(err, err_len, cudaGetErrorString(ce)); return MONA_ERR_CUDA; }

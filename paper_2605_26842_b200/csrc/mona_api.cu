@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <climits>
 #include <cmath>
 #include <cstdarg>
@@ -35,16 +36,21 @@ constexpr size_t WS_CTRL_BYTES = 1024 * 1024;        // per slot
 constexpr size_t CTRL_COUNTERS_OFF = 0;
 constexpr size_t CTRL_INVNORM_OFF = 4096;
 constexpr size_t CTRL_PARTIALS_OFF = 8192;
+constexpr size_t CTRL_SCHED_OFF = CTRL_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS;   // work counter + done counters of the NS kernel
 constexpr size_t WS_DATA_OFF = WS_CTRL_OFF + NSLOTS * WS_CTRL_BYTES;
-static_assert(CTRL_PARTIALS_OFF + sizeof(float) * MAXC * MAX_SLABS <= WS_CTRL_BYTES, "control block overflow");
+static_assert(CTRL_SCHED_OFF + sizeof(unsigned int) * (64 + (size_t)MAXC * NS_MAX_PHASES) <= WS_CTRL_BYTES, "control block overflow");
 static_assert(sizeof(unsigned int) * MAXC <= CTRL_INVNORM_OFF && sizeof(float) * MAXC <= CTRL_PARTIALS_OFF - CTRL_INVNORM_OFF, "control block overflow");
 
-// 1: consecutive chunks are pipelined over two streams; 0: everything runs on the caller's stream.
-int g_chunk_overlap = 1;
-
-// Bytes of bf16 iterates (X_t, X_{t+1}, A_t, B_t) a chunk may hold so that it stays resident in L2
-// between the 3T GEMMs of the iteration.
-size_t g_chunk_budget_bytes = 768ull << 20;
+// Process-wide defaults behind mona_set_chunk_budget() / mona_set_chunk_overlap().  They only seed
+// mona_default_options(); a handle keeps the options it was created with, so changing a default later
+// never reaches an existing handle.
+//   overlap: 1 = consecutive chunks are pipelined over two streams; 0 = everything on the caller's stream.
+//   budget : bytes of bf16 iterates (X_t, X_{t+1}, A_t, B'_t) one chunk may hold.  Chunks are sized to keep every
+//            SM pair busy, not for cache residency: chunks small enough to stay in L2 hold fewer tiles than the
+//            device has CTA pairs.
+constexpr size_t DEFAULT_CHUNK_BUDGET = 768ull << 20;
+std::atomic<int> g_chunk_overlap{1};
+std::atomic<size_t> g_chunk_budget_bytes{DEFAULT_CHUNK_BUDGET};
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -66,8 +72,9 @@ struct Bucket {
     size_t off_x[2] = {0, 0}, off_a = 0, off_b = 0;          // bf16 mode, bytes from the slot's iterate base
     size_t off32_x[2] = {0, 0}, off32_a = 0, off32_b = 0;    // fp32 mode
     size_t data_bytes = 0;
-    CUtensorMap tm_x[NSLOTS][2] = {}, tm_a[NSLOTS] = {}, tm_b[NSLOTS] = {};
+    NsMaps maps[NSLOTS] = {};      // per workspace slot: X ping, X pong, A, B' of a chunk of this bucket
 };
+constexpr int MAP_X0 = 0, MAP_A = 2, MAP_B = 3;
 
 struct Plan {
     std::vector<mona_matrix_desc> descs;
@@ -78,7 +85,7 @@ struct Plan {
     size_t state_bytes = 0, workspace_bytes = 0, slot_bytes = 0;
 };
 
-mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan, std::string& err) {
+mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, size_t chunk_budget, Plan& plan, std::string& err) {
     if (!descs || n_desc <= 0) { err = "descs is null or n_desc <= 0"; return MONA_ERR_INVALID_ARG; }
     plan.descs.assign(descs, descs + n_desc);
     std::map<std::tuple<int64_t, int64_t, int, int>, int> index;
@@ -123,14 +130,12 @@ mona_status build_plan(const mona_matrix_desc* descs, int64_t n_desc, Plan& plan
         b.off_A = state_bytes; state_bytes += align_up((size_t)count * b.e * aux, 256);
         b.off_G = state_bytes;                                              // the single-buffer form has no G_prev block
         if (b.state_dtype != MONA_STATE_COMBINED) state_bytes += align_up((size_t)count * b.e * aux, 256);
-        // slabs: ~16K elements each, at most MAX_SLABS, slab length a multiple of 1024
-        int64_t slab = 16384;
-        if ((b.e + slab - 1) / slab > MAX_SLABS) slab = (int64_t)align_up((size_t)((b.e + MAX_SLABS - 1) / MAX_SLABS), 1024);
+        long long slab = 0;
+        slab_plan(b.e, &slab, &b.slabs);
         b.slab_len = slab;
-        b.slabs = (int)((b.e + slab - 1) / slab);
         // chunk capacity
         const size_t per_mat_bf16 = (size_t)(2 * b.e + 2 * b.s * b.s) * 2;
-        int64_t cb = (int64_t)(g_chunk_budget_bytes / per_mat_bf16);
+        int64_t cb = (int64_t)(chunk_budget / per_mat_bf16);
         cb = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(cb, MAXC), count));
         b.Cb = (int)cb;
         b.Cf = (int)std::max<int64_t>(1, cb / 2);
@@ -177,6 +182,7 @@ F2 split(double v) {
 
 struct mona_handle {
     Plan plan;
+    mona_options opt = {};      // as resolved at creation; later changes of the process-wide defaults do not reach the handle
     int device = 0, max_pairs = 0;
     uint8_t* state = nullptr;
     uint8_t* ws = nullptr;
@@ -190,7 +196,7 @@ struct mona_handle {
     DeviceStatus* host_status = nullptr;   // pinned
     std::string last_error;
     int64_t launches = 0;
-    double flops_exec = 0.0, flops_dense = 0.0;
+    double flops_exec = 0.0, flops_dense = 0.0, flops_useful = 0.0;
 
     mona_status fail(mona_status st, const char* fmt, ...) {
         char buf[512];
@@ -222,32 +228,77 @@ mona_status mona_default_hparams(mona_hparams* hp) {
 
 mona_status mona_set_chunk_budget(size_t bytes) {
     if (bytes < (1u << 20)) return MONA_ERR_INVALID_ARG;
-    g_chunk_budget_bytes = bytes;
+    g_chunk_budget_bytes.store(bytes);
     return MONA_OK;
 }
 
 mona_status mona_set_chunk_overlap(int enabled) {
-    g_chunk_overlap = enabled ? 1 : 0;
+    g_chunk_overlap.store(enabled ? 1 : 0);
     return MONA_OK;
 }
 
-mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc, size_t* state_bytes, size_t* workspace_bytes) {
+mona_status mona_default_options(mona_options* opt) {
+    if (!opt) return MONA_ERR_INVALID_ARG;
+    memset(opt, 0, sizeof *opt);
+    opt->chunk_budget_bytes = g_chunk_budget_bytes.load();
+    opt->chunk_overlap = g_chunk_overlap.load();
+    opt->fuse_update = 1;
+    opt->ns_delay = 3;
+    return MONA_OK;
+}
+
+}  // extern "C"
+
+namespace {
+// Options as the plan uses them: NULL means the defaults; a zero budget or delay means the default value.
+mona_status resolve_options(const mona_options* in, mona_options& out) {
+    mona_default_options(&out);
+    if (!in) return MONA_OK;
+    if (in->chunk_budget_bytes != 0) {
+        if (in->chunk_budget_bytes < (1u << 20)) return MONA_ERR_INVALID_ARG;
+        out.chunk_budget_bytes = in->chunk_budget_bytes;
+    }
+    out.chunk_overlap = in->chunk_overlap ? 1 : 0;
+    out.fuse_update = in->fuse_update ? 1 : 0;
+    if (in->ns_delay < 0 || in->ns_delay > 64) return MONA_ERR_INVALID_ARG;
+    if (in->ns_delay > 0) out.ns_delay = in->ns_delay;
+    return MONA_OK;
+}
+}  // namespace
+
+extern "C" {
+
+mona_status mona_query_sizes_opt(const mona_matrix_desc* descs, int64_t n_desc, const mona_options* options,
+                                 size_t* state_bytes, size_t* workspace_bytes) {
+    mona_options opt;
+    if (resolve_options(options, opt) != MONA_OK) return MONA_ERR_INVALID_ARG;
     Plan plan;
     std::string err;
-    mona_status st = build_plan(descs, n_desc, plan, err);
+    mona_status st = build_plan(descs, n_desc, opt.chunk_budget_bytes, plan, err);
     if (st != MONA_OK) return st;
     if (state_bytes) *state_bytes = plan.state_bytes;
     if (workspace_bytes) *workspace_bytes = plan.workspace_bytes;
     return MONA_OK;
 }
 
+mona_status mona_query_sizes(const mona_matrix_desc* descs, int64_t n_desc, size_t* state_bytes, size_t* workspace_bytes) {
+    return mona_query_sizes_opt(descs, n_desc, nullptr, state_bytes, workspace_bytes);
+}
+
 mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc, void* state, size_t state_bytes,
                         void* workspace, size_t workspace_bytes, int device) {
+    return mona_create_opt(out, descs, n_desc, nullptr, state, state_bytes, workspace, workspace_bytes, device);
+}
+
+mona_status mona_create_opt(mona_handle** out, const mona_matrix_desc* descs, int64_t n_desc, const mona_options* options,
+                            void* state, size_t state_bytes, void* workspace, size_t workspace_bytes, int device) {
     if (!out) return MONA_ERR_INVALID_ARG;
     *out = nullptr;
     mona_handle* h = new mona_handle();
     *out = h;     // returned even on failure so that mona_last_error() can be read; destroy it either way
-    mona_status st = build_plan(descs, n_desc, h->plan, h->last_error);
+    if (resolve_options(options, h->opt) != MONA_OK)
+        return h->fail(MONA_ERR_INVALID_ARG, "options: chunk_budget_bytes must be 0 or at least 1 MiB, ns_delay within 0..64");
+    mona_status st = build_plan(descs, n_desc, h->opt.chunk_budget_bytes, h->plan, h->last_error);
     if (st != MONA_OK) return st;
     if (!state || !workspace) return h->fail(MONA_ERR_INVALID_ARG, "state or workspace is null");
     if (((uintptr_t)state & 255) || ((uintptr_t)workspace & 255)) return h->fail(MONA_ERR_ALIGNMENT, "state/workspace must be 256-byte aligned");
@@ -274,13 +325,13 @@ mona_status mona_create(mona_handle** out, const mona_matrix_desc* descs, int64_
         bool ok = true;
         for (int sl = 0; sl < NSLOTS; ++sl) {
             uint8_t* data = h->ws + WS_DATA_OFF + sl * h->plan.slot_bytes;
-            for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.tm_x[sl][i], data + b.off_x[i], b.cols, b.rows, b.Cb);
-            ok = ok && encode_map(encode, &b.tm_a[sl], data + b.off_a, b.s, b.s, b.Cb);
-            ok = ok && encode_map(encode, &b.tm_b[sl], data + b.off_b, b.s, b.s, b.Cb);
+            for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.maps[sl].m[MAP_X0 + i], data + b.off_x[i], b.cols, b.rows, b.Cb);
+            ok = ok && encode_map(encode, &b.maps[sl].m[MAP_A], data + b.off_a, b.s, b.s, b.Cb);
+            ok = ok && encode_map(encode, &b.maps[sl].m[MAP_B], data + b.off_b, b.s, b.s, b.Cb);
         }
         if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
     }
-    MONA_CUDA(h, tc_gemm_configure(&h->max_pairs));
+    MONA_CUDA(h, ns_configure(&h->max_pairs));
     MONA_CUDA(h, small_ns_configure());
     MONA_CUDA(h, cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking));
     MONA_CUDA(h, cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming));
@@ -335,7 +386,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
         const int capb = tcb ? b.Cb : b.Cf;
         total_chunks += ((int64_t)b.mats.size() + capb - 1) / capb;
     }
-    const bool overlap = g_chunk_overlap && total_chunks > 1;
+    const bool overlap = h->opt.chunk_overlap && total_chunks > 1;
     cudaStream_t slot_stream[NSLOTS] = {(cudaStream_t)stream_v, overlap ? h->side : (cudaStream_t)stream_v};
     if (overlap) {
         MONA_CUDA(h, cudaEventRecord(h->ev_fork, slot_stream[0]));
@@ -347,6 +398,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
     h->launches = 0;
     h->flops_exec = 0.0;
     h->flops_dense = 0.0;
+    h->flops_useful = 0.0;
 
     for (const Bucket& b : plan.buckets) {
         const bool tc = (hp->ns_precision == 0) && b.tc_ok && T >= 1;
@@ -400,38 +452,53 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                 ++h->launches;
             }
             const void* o_final = nullptr;
+            bool update_fused = false;
             if (tc) {
                 if (phase_mask & 2u) {
-                    for (int t = 0; t < T; ++t) {
-                        const int cur = t & 1, nxt = cur ^ 1;
-                        TcGemm g1{};     // A = X X^T (wide) or X^T X (tall): lower-triangle tiles only
-                        g1.C = C; g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_mn = g1.b_mn = b.tall ? 1 : 0; g1.symmetric = 1; g1.ab_same = 1;
-                        g1.cin = nullptr; g1.c1 = 0.f; g1.c2 = 1.f;
-                        g1.inv_norm = inv_norm; g1.post_mode = t == 0 ? 2 : 0;
-                        tc_gemm_plan(g1);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_x[slot][cur], b.tm_x[slot][cur], b.tm_a[slot], g1, h->max_pairs, dstatus, stream));
-                        TcGemm g2{};     // B' = b A + c A A + a I, operands and result lower-block-stored
-                        g2.C = C; g2.M = g2.N = g2.K = (int)b.s; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
-                        g2.cin = ab; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c;
-                        g2.inv_norm = inv_norm; g2.post_mode = 0; g2.diag_add = ns_a;
-                        tc_gemm_plan(g2);
-                        MONA_CUDA(h, launch_tc_gemm(b.tm_a[slot], b.tm_a[slot], b.tm_b[slot], g2, h->max_pairs, dstatus, stream));
-                        TcGemm g3{};
-                        g3.C = C; g3.K = (int)b.s; g3.symmetric = 0; g3.wide = 1;   // 256 x 512 macro-tiles
-                        g3.cin = nullptr; g3.c1 = 0.f; g3.c2 = 1.f;
-                        g3.inv_norm = inv_norm; g3.post_mode = t == 0 ? 1 : 0;
-                        if (!b.tall) {   // X' = B' X : B' is the symmetric "A" operand, X the MN-major "B" operand
-                            g3.M = (int)b.s; g3.N = (int)b.l; g3.a_sym = 1; g3.b_mn = 1;
-                            tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_b[slot], b.tm_x[slot][cur], b.tm_x[slot][nxt], g3, h->max_pairs, dstatus, stream));
-                        } else {         // X' = X B' : X is K-major, the symmetric B' serves as its own transpose
-                            g3.M = (int)b.l; g3.N = (int)b.s; g3.a_mn = 0; g3.b_sym = 1;
-                            tc_gemm_plan(g3);
-                            MONA_CUDA(h, launch_tc_gemm(b.tm_x[slot][cur], b.tm_b[slot], b.tm_x[slot][nxt], g3, h->max_pairs, dstatus, stream));
+                    // the last X' = B' X applies the parameter update in its epilogue when this call runs both phases and the
+                    // fp32 rows can be accessed 32 bytes at a time
+                    update_fused = h->opt.fuse_update && (phase_mask & 4u) != 0u;
+                    for (int c = 0; c < C && update_fused; ++c)
+                        if (((uintptr_t)ptrs.w[c] & 31) || ((uintptr_t)ptrs.o[c] & 31)) update_fused = false;
+                    unsigned int* sched = (unsigned int*)(ctrl + CTRL_SCHED_OFF);
+                    __nv_bfloat16* bb = (__nv_bfloat16*)(data + b.off_b);
+                    for (int t0 = 0; t0 < T; t0 += NS_MAX_PHASES / 3) {
+                        const int t1 = std::min(T, t0 + NS_MAX_PHASES / 3);
+                        NsProgram g{};
+                        g.C = C; g.P = 3 * (t1 - t0); g.delay = h->opt.ns_delay;
+                        g.inv_norm = inv_norm; g.work_counter = sched; g.done = sched + 64;
+                        g.eta_lambda = eta_lambda; g.eta_gamma = eta_gamma;
+                        for (int t = t0; t < t1; ++t) {
+                            const int cur = t & 1, nxt = cur ^ 1;
+                            NsPhase& g1 = g.ph[3 * (t - t0)];      // A = X X^T (wide) or X^T X (tall): lower-triangle tiles only
+                            g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_map = g1.b_map = MAP_X0 + cur; g1.a_mn = g1.b_mn = b.tall ? 1 : 0;
+                            g1.symmetric = 1; g1.ab_same = 1; g1.d = ab; g1.ld = b.s; g1.mat_stride = b.s * b.s;
+                            g1.c1 = 0.f; g1.c2 = 1.f; g1.post_mode = t == 0 ? 2 : 0;
+                            ns_phase_plan(g1);
+                            NsPhase& g2 = g.ph[3 * (t - t0) + 1];  // B' = b A + c A A + a I, operands and result lower-block-stored
+                            g2.M = g2.N = g2.K = (int)b.s; g2.a_map = g2.b_map = MAP_A; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
+                            g2.cin = ab; g2.d = bb; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c; g2.diag_add = ns_a;
+                            ns_phase_plan(g2);
+                            NsPhase& g3 = g.ph[3 * (t - t0) + 2];  // X' = B' X (wide) or X B' (tall), 256 x 512 macro-tiles
+                            g3.K = (int)b.s; g3.wide = 1; g3.d = xb[nxt]; g3.ld = b.cols; g3.mat_stride = b.e;
+                            g3.c1 = 0.f; g3.c2 = 1.f; g3.post_mode = t == 0 ? 1 : 0;
+                            g3.fuse_update = (update_fused && t == T - 1) ? 1 : 0;
+                            if (!b.tall) {   // B' is the symmetric "A" operand, X the MN-major "B" operand
+                                g3.M = (int)b.s; g3.N = (int)b.l; g3.a_map = MAP_B; g3.a_sym = 1; g3.b_map = MAP_X0 + cur; g3.b_mn = 1;
+                            } else {         // X is K-major, the symmetric B' serves as its own transpose
+                                g3.M = (int)b.l; g3.N = (int)b.s; g3.a_map = MAP_X0 + cur; g3.a_mn = 0; g3.b_map = MAP_B; g3.b_sym = 1;
+                            }
+                            ns_phase_plan(g3);
+                            h->flops_exec += (double)C * (ns_phase_executed_flops(g1) + ns_phase_executed_flops(g2) + ns_phase_executed_flops(g3));
+                            h->flops_dense += (double)C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
+                            h->flops_useful += (double)C * (3.0 * b.s * b.s * b.l + (double)b.s * b.s * b.s);
                         }
-                        h->launches += 3;
-                        h->flops_exec += tc_gemm_executed_flops(g1) + tc_gemm_executed_flops(g2) + tc_gemm_executed_flops(g3);
-                        h->flops_dense += (double)C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
+                        ns_program_plan(g);
+                        MONA_CUDA(h, cudaMemsetAsync(sched, 0, sizeof(unsigned int) * ns_sched_words(C, g.P), stream));
+                        NsUpdatePtrs up{};
+                        if (update_fused && t1 == T) { up.w = ptrs.w; up.o = ptrs.o; }
+                        MONA_CUDA(h, launch_ns_program(b.maps[slot], g, up, h->max_pairs, dstatus, stream));
+                        ++h->launches;
                     }
                 }
                 o_final = xb[T & 1];
@@ -481,7 +548,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                 }
                 o_final = xf[T & 1];
             }
-            if (phase_mask & 4u) {
+            if ((phase_mask & 4u) && !update_fused) {
                 MONA_CUDA(h, launch_update(ptrs, C, tc, vec4, o_final, b.e, b.slab_len, b.slabs, eta_lambda, eta_gamma, stream));
                 ++h->launches;
             }
@@ -557,10 +624,14 @@ mona_status mona_step_host(mona_handle* h, const mona_hparams* hp, void* const* 
         }
     }
     mona_status st = step_impl(h, hp, params, (const void* const*)grads, nullptr, 7u, stream_v, params_host);
-    if (st != MONA_OK) return st;
+    // join the copy streams back into the caller's stream whether or not the step was enqueued completely
+    const std::string step_error = h->last_error;
+    MONA_CUDA(h, cudaEventRecord(h->ev_hjoin, h->h2d));
+    MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_hjoin, 0));
     MONA_CUDA(h, cudaEventRecord(h->ev_hjoin, h->d2h));
     MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_hjoin, 0));
-    return MONA_OK;
+    if (st != MONA_OK) h->last_error = step_error;
+    return st;
 }
 
 mona_status mona_selftest_timeout(mona_handle* h, void* stream_v) {
@@ -568,13 +639,20 @@ mona_status mona_selftest_timeout(mona_handle* h, void* stream_v) {
     MONA_CUDA(h, cudaSetDevice(h->device));
     for (const Bucket& b : h->plan.buckets) {
         if (!b.tc_ok) continue;
-        // one X X^T launch over the first matrix slot of the workspace whose stages expect 16 bytes too many
-        TcGemm g{};
-        g.C = 1; g.M = g.N = (int)b.s; g.K = (int)b.l; g.a_mn = g.b_mn = b.tall ? 1 : 0; g.symmetric = 1; g.ab_same = 1;
-        g.c1 = 0.f; g.c2 = 1.f; g.inv_norm = (const float*)(h->ws + WS_CTRL_OFF + CTRL_INVNORM_OFF); g.post_mode = 0;
+        // one X X^T phase over the first matrix slot of the workspace whose stages expect 16 bytes too many
+        uint8_t* ctrl = h->ws + WS_CTRL_OFF;
+        uint8_t* data = h->ws + WS_DATA_OFF;
+        unsigned int* sched = (unsigned int*)(ctrl + CTRL_SCHED_OFF);
+        NsProgram g{};
+        g.C = 1; g.P = 1; g.delay = 1; g.inv_norm = (const float*)(ctrl + CTRL_INVNORM_OFF); g.work_counter = sched; g.done = sched + 64;
         g.selftest_extra_tx = 16;
-        tc_gemm_plan(g);
-        MONA_CUDA(h, launch_tc_gemm(b.tm_x[0][0], b.tm_x[0][0], b.tm_a[0], g, h->max_pairs, (DeviceStatus*)(h->ws + WS_STATUS_OFF), (cudaStream_t)stream_v));
+        NsPhase& p = g.ph[0];
+        p.M = p.N = (int)b.s; p.K = (int)b.l; p.a_map = p.b_map = MAP_X0; p.a_mn = p.b_mn = b.tall ? 1 : 0; p.symmetric = 1; p.ab_same = 1;
+        p.d = (__nv_bfloat16*)(data + b.off_a); p.ld = b.s; p.mat_stride = b.s * b.s; p.c1 = 0.f; p.c2 = 1.f;
+        ns_phase_plan(p);
+        ns_program_plan(g);
+        MONA_CUDA(h, cudaMemsetAsync(sched, 0, sizeof(unsigned int) * ns_sched_words(1, 1), (cudaStream_t)stream_v));
+        MONA_CUDA(h, launch_ns_program(b.maps[0], g, NsUpdatePtrs{}, h->max_pairs, (DeviceStatus*)(h->ws + WS_STATUS_OFF), (cudaStream_t)stream_v));
         return MONA_OK;
     }
     return h->fail(MONA_ERR_UNSUPPORTED_SHAPE, "no descriptor of this handle takes the tensor-core path");
@@ -612,6 +690,12 @@ mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* d
     if (!h) return MONA_ERR_INVALID_ARG;
     if (executed) *executed = h->flops_exec;
     if (dense_equivalent) *dense_equivalent = h->flops_dense;
+    return MONA_OK;
+}
+
+mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful) {
+    if (!h || !useful) return MONA_ERR_INVALID_ARG;
+    *useful = h->flops_useful;
     return MONA_OK;
 }
 

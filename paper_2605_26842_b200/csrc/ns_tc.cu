@@ -1,68 +1,65 @@
-// Tensor-core GEMMs of the Newton-Schulz iteration (Eq. newton_schulz) for sm_100a.
+// Tensor-core Newton-Schulz iteration (Eq. newton_schulz) for sm_100a: ONE persistent kernel per chunk runs
+// every GEMM of up to five iterations - A = X X^T, B' = b A + c A^2 + a I, X' = B' X - over all matrices of
+// the chunk.
 //
-// The kernel is persistent and runs as clusters of two CTAs on neighbouring SMs.  A CTA pair walks a
-// static list of 256 x 256 output tiles of all matrices of a chunk; one tcgen05.mma.cta_group::2
-// instruction stream, issued by the even CTA (the "leader"), drives the tensor cores of both SMs.
-// Each CTA stages its own 128 rows of the A operand and its own 128 rows of the B operand per k-slice,
-// so a pair moves 64 KiB from L2 per 256 x 256 x 64 step (half of what two independent 128 x 256 tiles
-// would).  Roles inside a CTA:
-//   warp 0     TMA producer: operand boxes into a ring of shared-memory stages; the copies of both CTAs
+// Work items are 256 x 256 output tiles (256 x 512 macro-tiles for X' = B' X).  They are handed out through
+// one atomic counter, in an order in which every item follows the items it depends on, and the phase-to-phase
+// dependency of a matrix is a counter in global memory: the pair that takes phase q of matrix c waits until
+// all items of phase q - 1 of matrix c have been stored.  Because a waiting pair only waits for items that
+// running pairs already hold, the scheme cannot deadlock whatever share of the grid is resident.  There is no
+// launch boundary, no partial last wave and no static tile assignment between the GEMMs of a chunk; the
+// intermediate matrices are consumed a few hundred microseconds after they were produced.
+//
+// The kernel runs as clusters of two CTAs on neighbouring SMs; one tcgen05.mma.cta_group::2 instruction
+// stream, issued by the even CTA (the "leader"), drives the tensor cores of both SMs.  Each CTA stages its own
+// 128 rows of the A operand and its own 128 rows of the B operand per k-slice, so a pair moves 64 KiB from L2
+// per 256 x 256 x 64 step (half of what two independent 128 x 256 tiles would).  Roles inside a CTA:
+//   warp 0     lane 0 of the leader: scheduler (takes items, waits for their dependencies, publishes them to
+//              both CTAs through a small ring in shared memory) and TMA producer; lane 0 of the peer: TMA
+//              producer.  Operand boxes go into a ring of shared-memory stages; the copies of both CTAs
 //              complete on the leader's "full" barrier,
 //   warp 1     owner of tensor memory; in the leader its lane 0 issues the MMAs and commits them to
 //              the "empty" barriers of both CTAs (multicast commit),
 //   warps 2-9  epilogue: tcgen05.ld the CTA's 128 x 256 fp32 accumulator, apply the polynomial term
-//              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, pack to bf16 into swizzled
-//              shared memory and hand the boxes to TMA stores.
-// Tensor memory holds two 256-column accumulators.  In the plain configuration they alternate, so the
-// epilogue of one tile overlaps the main loop of the next.  In the WIDE configuration (non-symmetric
-// products, here X' = B' X) a pair computes a 256 x 512 macro-tile, i.e. two neighbouring tiles at once,
-// one per accumulator, from ONE staged slice of the A operand: 96 KiB instead of 128 KiB cross from L2
-// per k-slice and pair.  The main loop is bound by that traffic, not by the tensor pipe, so fewer bytes
-// per flop is worth more than accumulator double-buffering.  To keep the unhidden part of that epilogue short,
-// its warps first read and pack a whole accumulator into registers and hand it back to the MMA issuer, and only
-// then stage and store; the operand ring keeps filling meanwhile.
+//              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, and store bf16 rows straight from
+//              registers (each thread owns 64 consecutive columns of one row, i.e. whole 128-byte lines);
+//              for the last X' = B' X of a step the same warps apply the parameter update of Eq. muon_update
+//              to the fp32 weights instead.  Then they count the item as done.
+// Tensor memory holds two 256-column accumulators.  Plain tiles alternate between them, so the epilogue of one
+// tile overlaps the main loop of the next.  A macro-tile uses both at once, two neighbouring tiles computed
+// from ONE staged slice of the A operand: 96 KiB instead of 128 KiB cross from L2 per k-slice and pair.
 //
-// Every wait on an mbarrier is bounded: when one runs out the CTA latches STATUS_TIMEOUT, raises its
-// abort flag, and all roles fall through to the common exit, where tensor memory is released.
+// Every wait - on an mbarrier or on a dependency counter - is bounded: when one runs out the CTA latches
+// STATUS_TIMEOUT, raises its abort flag, and all roles fall through to the common exit, where tensor memory
+// is released.
 #include "ns_tc.cuh"
 
 namespace mona {
 
 namespace {
 
-#ifndef MONA_TC_WIDE_STAGES
-#define MONA_TC_WIDE_STAGES 4
-#endif
-#ifndef MONA_TC_WIDE_EPI_BUFS
-#define MONA_TC_WIDE_EPI_BUFS 1
-#endif
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
 constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
-// 320 threads x 160 registers: no spills, and room is left on the SM for one 256-thread block of another kernel
-constexpr int TC_MAX_REGS = 160;
+// registers are granted to warps in groups of four: 10 warps count as 12, and 12 x 32 x 168 fits the SM's 64 K
+constexpr int TC_MAX_REGS = 168;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
 constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
 constexpr uint32_t A_STAGE_BYTES = CTA_M * TC_BK * 2;             // 16 KiB
 constexpr uint32_t B_SUB_BYTES = CTA_N * TC_BK * 2;               // 16 KiB per 256-column tile
 constexpr int EPI_COLS = 128;                                     // output columns per epilogue phase
-constexpr uint32_t EPI_BUF_BYTES = CTA_M * EPI_COLS * 2;          // 32 KiB = 2 x 2 boxes
 constexpr uint32_t TMEM_COLS = 512;                               // 2 accumulators x 256 fp32 columns
-constexpr uint32_t SMEM_CTRL_BYTES = 256;
+constexpr int STAGES = 4;                                         // operand ring depth
+constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + 2 * B_SUB_BYTES; // 48 KiB: room for a macro-tile's k-slice
+constexpr int RING = 4;                                           // published-but-unfinished work items
+constexpr uint32_t SMEM_CTRL_BYTES = 512;
+constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_CTRL_BYTES + 1024;
 constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
-
-// Shared-memory plan of the two configurations (per CTA).
-template <bool WIDE>
-struct Cfg {
-    static constexpr int NSUB = WIDE ? 2 : 1;                                   // 256-column tiles per macro-tile
-    static constexpr int STAGES = WIDE ? MONA_TC_WIDE_STAGES : 5;               // operand ring depth
-    static constexpr int EPI_BUFS = WIDE ? MONA_TC_WIDE_EPI_BUFS : 2;           // staging buffers of the store epilogue
-    static constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + NSUB * B_SUB_BYTES; // 48 / 32 KiB
-    static constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
-    static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-    static_assert(8 * (2 * STAGES + 4) + 8 <= SMEM_CTRL_BYTES, "control block");
-};
+// readers of a published item: MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
+constexpr uint32_t RING_READERS = 1 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
+static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
+static_assert(8 * (2 * STAGES + 4 + 2 * RING) + 16 + 16 * RING <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -91,20 +88,25 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
-// Arrive on a barrier given by its cluster-wide address (own CTA or the peer).
+// Arrive (release at cluster scope) on a barrier given by its cluster-wide address (own CTA or the peer).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ void latch_timeout(volatile int* abort_flag, DeviceStatus* status, unsigned site) {
+    *abort_flag = 1;
+    atomicOr(&status->flags, STATUS_TIMEOUT);
+    status->timeout_site = site;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
@@ -117,9 +119,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
-                *abort_flag = 1;
-                atomicOr(&status->flags, STATUS_TIMEOUT);
-                status->timeout_site = site;
+                latch_timeout(abort_flag, status, site);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned int* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Bounded wait until a dependency counter in global memory has reached `need` (acquire at device scope).
+__device__ __forceinline__ bool wait_counter(const unsigned int* ctr, unsigned need, volatile int* abort_flag,
+                                             DeviceStatus* status, unsigned site) {
+    if (ld_acquire_gpu(ctr) >= need) return true;
+    const long long t0 = clock64();
+    unsigned spins = 0;
+    while (true) {
+        if (ld_acquire_gpu(ctr) >= need) return true;
+        __nanosleep(64);
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
+                latch_timeout(abort_flag, status, site);
                 return false;
             }
         }
@@ -153,16 +176,9 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
-                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Orders this thread's earlier generic-proxy accesses (plain loads/stores, acquire loads) with later accesses
+// through the asynchronous proxy (TMA), and the other way round.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // ---- tcgen05 --------------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
@@ -233,30 +249,32 @@ __device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn) {
            | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
-struct TileCoord {
-    int c, tm, tn;   // matrix, tile row, first tile column
-    int nsub;        // 256-column tiles in this (macro-)tile: 1 or 2
+// A published work item: item `t` of phase `q` for matrix `c`; stop != 0 ends the role loops.
+struct Item {
+    int c, q, t, stop;
 };
 
-template <bool WIDE>
-__device__ __forceinline__ TileCoord decode_tile(const TcGemm& g, int t) {
+struct TileCoord {
+    int tm, tn;      // tile row, first tile column
+    int nsub;        // 256-column tiles in this item: 1 or 2
+};
+
+__device__ __forceinline__ TileCoord decode_tile(const NsPhase& p, int r) {
     TileCoord tc;
-    tc.c = t / g.tiles_per_mat;
-    const int r = t - tc.c * g.tiles_per_mat;
     tc.nsub = 1;
-    if (WIDE) {
-        const int macro_n = (g.tiles_n + 1) >> 1;
+    if (p.wide) {
+        const int macro_n = (p.tiles_n + 1) >> 1;
         tc.tm = r / macro_n;
         tc.tn = 2 * (r - tc.tm * macro_n);
-        tc.nsub = tc.tn + 1 < g.tiles_n ? 2 : 1;
-    } else if (g.symmetric) {
+        tc.nsub = tc.tn + 1 < p.tiles_n ? 2 : 1;
+    } else if (p.symmetric) {
         int tm = 0;
         while ((tm + 1) * (tm + 2) / 2 <= r) ++tm;     // lower triangle, row by row
         tc.tm = tm;
         tc.tn = r - tm * (tm + 1) / 2;
     } else {
-        tc.tm = r / g.tiles_n;
-        tc.tn = r - tc.tm * g.tiles_n;
+        tc.tm = r / p.tiles_n;
+        tc.tn = r - tc.tm * p.tiles_n;
     }
     return tc;
 }
@@ -275,40 +293,54 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
     return r;
 }
 
-template <bool WIDE>
+// 32-byte accesses to fp32 rows (the parameter update of the fused epilogue)
+__device__ __forceinline__ void ld8(const float* p, float* v) {
+    asm volatile("ld.global.cs.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void st8(float* p, const float* v) {
+    asm volatile("st.global.cs.v8.f32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};"
+                 ::"f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p)
+                 : "memory");
+}
+
+// Per-matrix pointers of the fused parameter update, passed by value (all null when no phase fuses it).
+struct UpdateTable {
+    float* w[MAXC];
+    float* o[MAXC];
+};
+
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(TC_MAX_REGS)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant__ CUtensorMap tma_b,
-               const __grid_constant__ CUtensorMap tma_d, TcGemm g, DeviceStatus* __restrict__ status) {
-    using C = Cfg<WIDE>;
-    constexpr int STAGES = C::STAGES;
-    constexpr uint32_t STAGE_BYTES = C::STAGE_BYTES;
+ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsProgram g,
+                const __grid_constant__ UpdateTable upd, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzle atoms need 1024-byte alignment
-    const uint32_t epi_base = base + STAGES * STAGE_BYTES;
-    const uint32_t ctrl = epi_base + C::EPI_BUFS * EPI_BUF_BYTES;
+    const uint32_t ctrl = base + STAGES * STAGE_BYTES;
     const uint32_t bar_full = ctrl;                             // STAGES x 8 B (used in the leader)
-    const uint32_t bar_empty = ctrl + 8 * STAGES;               // STAGES x 8 B
-    const uint32_t bar_acc_full = ctrl + 16 * STAGES;           // 2 x 8 B, one per accumulator
+    const uint32_t bar_empty = bar_full + 8 * STAGES;           // STAGES x 8 B
+    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;       // 2 x 8 B, one per accumulator
     const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B (used in the leader)
-    const uint32_t tmem_slot = bar_acc_empty + 16;              // 4 B
+    const uint32_t bar_ring_full = bar_acc_empty + 16;          // RING x 8 B
+    const uint32_t bar_ring_empty = bar_ring_full + 8 * RING;   // RING x 8 B (used in the leader)
+    const uint32_t tmem_slot = bar_ring_empty + 8 * RING;       // 4 B + abort flag 4 B + 8 B pad
+    const uint32_t ring_items = tmem_slot + 16;                 // RING x 16 B
     uint8_t* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + (tmem_slot - ctrl));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + (tmem_slot - ctrl) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                    // 0: leader, 1: peer
-    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int total_tiles = g.C * g.tiles_per_mat;
-    const int num_kb = (g.K + TC_BK - 1) / TC_BK;
+    const int P = g.P;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
+        for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_a) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_b) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tma_d) : "memory");
+        #pragma unroll
+        for (int i = 0; i < NS_MAPS; ++i) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[i]) : "memory");
     }
     if (warp == 1) {
         __syncwarp();
@@ -321,50 +353,116 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
 
-    // Accumulator of sub-tile j of the n-th (macro-)tile this pair processes: WIDE uses accumulator j,
-    // the plain configuration alternates.  Every role keeps one use-parity bit per accumulator.
+    // A reader's view of the item ring: wait for the n-th published item, copy it, hand the slot back.
+    const uint32_t ring_empty_leader = map_to_cta(bar_ring_empty, 0);
+    auto take_item = [&](unsigned n, Item& it, unsigned site, bool arrive) -> bool {
+        const uint32_t slot = n % RING, par = (n / RING) & 1u;
+        if (!mbar_wait(bar_ring_full + 8 * slot, par, abort_flag, status, site)) return false;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(it.c), "=r"(it.q), "=r"(it.t), "=r"(it.stop) : "r"(ring_items + 16 * slot) : "memory");
+        if (arrive) mbar_arrive_cluster(ring_empty_leader + 8 * slot);
+        return true;
+    };
 
-    if (warp == 0) {
-        // ---------------- TMA producer (both CTAs) ----------------
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            bool ok = true;
-            const uint32_t full_leader = map_to_cta(bar_full, 0);
-            for (int t = pair; t < total_tiles && ok; t += num_pairs) {
-                const TileCoord tc = decode_tile<WIDE>(g, t);
-                const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;      // this CTA's rows of the A operand
-                const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand (first sub-tile)
-                // diagonal tile of X X^T or A A: both operands are the same rows, staged once
-                const bool shared_ab = !WIDE && g.ab_same && tc.tm == tc.tn;
-                const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (shared_ab ? 0u : (uint32_t)tc.nsub * B_SUB_BYTES)) + (uint32_t)g.selftest_extra_tx;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!(ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1))) break;
-                    const uint32_t full = full_leader + 8 * stage;
-                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-                    const int k0 = kb * TC_BK;
-                    if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx_bytes);   // both CTAs' copies land here
-                    const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
+    // TMA loads of all k-slices of one item into the stage ring (both CTAs run this, each for its own rows).
+    uint32_t stage = 0, phase = 0;
+    const uint32_t full_leader = map_to_cta(bar_full, 0);
+    auto produce = [&](const Item& it) -> bool {
+        const NsPhase& p = g.ph[it.q];
+        const TileCoord tc = decode_tile(p, it.t);
+        const CUtensorMap* tma_a = &maps.m[p.a_map];
+        const CUtensorMap* tma_b = &maps.m[p.b_map];
+        const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;      // this CTA's rows of the A operand
+        const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand (first sub-tile)
+        // diagonal tile of X X^T or A A: both operands are the same rows, staged once
+        const bool shared_ab = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
+        const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (shared_ab ? 0u : (uint32_t)tc.nsub * B_SUB_BYTES)) + (uint32_t)g.selftest_extra_tx;
+        const int num_kb = (p.K + TC_BK - 1) / TC_BK;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1)) return false;
+            const uint32_t full = full_leader + 8 * stage;
+            const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+            const int k0 = kb * TC_BK;
+            if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx_bytes);   // both CTAs' copies land here
+            const int a_mn = p.a_sym ? fetch_transposed(1, tc.tm, k0) : p.a_mn;
+            #pragma unroll
+            for (int j = 0; j < CTA_M / TC_BOX; ++j) {
+                if (a_mn) tma_load_3d(sa + j * BOX_BYTES, tma_a, full, m0 + j * TC_BOX, k0, it.c);
+                else      tma_load_3d(sa + j * BOX_BYTES, tma_a, full, k0, m0 + j * TC_BOX, it.c);
+            }
+            if (!shared_ab) {
+                for (int u = 0; u < tc.nsub; ++u) {
+                    const int b_mn = p.b_sym ? fetch_transposed(1, tc.tn + u, k0) : p.b_mn;
+                    const int nu = n0 + u * TC_BN;
+                    const uint32_t sbu = sb + u * B_SUB_BYTES;
                     #pragma unroll
-                    for (int j = 0; j < CTA_M / TC_BOX; ++j) {
-                        if (a_mn) tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, m0 + j * TC_BOX, k0, tc.c);
-                        else      tma_load_3d(sa + j * BOX_BYTES, &tma_a, full, k0, m0 + j * TC_BOX, tc.c);
+                    for (int j = 0; j < CTA_N / TC_BOX; ++j) {
+                        if (b_mn) tma_load_3d(sbu + j * BOX_BYTES, tma_b, full, nu + j * TC_BOX, k0, it.c);
+                        else      tma_load_3d(sbu + j * BOX_BYTES, tma_b, full, k0, nu + j * TC_BOX, it.c);
                     }
-                    if (!shared_ab) {
-                        for (int u = 0; u < tc.nsub; ++u) {
-                            const int b_mn = g.b_sym ? fetch_transposed(1, tc.tn + u, k0) : g.b_mn;
-                            const int nu = n0 + u * TC_BN;
-                            const uint32_t sbu = sb + u * B_SUB_BYTES;
-                            #pragma unroll
-                            for (int j = 0; j < CTA_N / TC_BOX; ++j) {
-                                if (b_mn) tma_load_3d(sbu + j * BOX_BYTES, &tma_b, full, nu + j * TC_BOX, k0, tc.c);
-                                else      tma_load_3d(sbu + j * BOX_BYTES, &tma_b, full, k0, nu + j * TC_BOX, tc.c);
-                            }
-                        }
-                    }
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        return true;
+    };
+
+    if (warp == 0) {
+        if (lane == 0 && rank == 0) {
+            // ---------------- scheduler + TMA producer (leader) ----------------
+            const uint32_t ring_items_peer = map_to_cta(ring_items, 1), ring_full_peer = map_to_cta(bar_ring_full, 1);
+            const uint32_t ring_full_own = map_to_cta(bar_ring_full, 0);
+            int cur_tau = 0, cur_q = 0;                // group (tau, q) of the item order the cursor stands in
+            unsigned cur_base = 0;                     // index of the first item of that group
+            unsigned published = 0;
+            unsigned idx = atomicAdd(g.work_counter, 1u);
+            bool ok = true;
+            while (ok) {
+                Item it;
+                it.c = it.q = it.t = 0;
+                it.stop = idx >= g.total_items ? 1 : 0;
+                unsigned next_idx = 0;
+                if (!it.stop) {
+                    next_idx = atomicAdd(g.work_counter, 1u);      // in flight while this item is being staged
+                    // item order: for tau = 0, 1, ...: for q = 0 .. P-1: matrix c = tau - delay * q (if it exists): its items
+                    while (true) {
+                        const int c = cur_tau - g.delay * cur_q;
+                        const unsigned n = (c >= 0 && c < g.C) ? (unsigned)g.ph[cur_q].items_per_mat : 0u;
+                        if (idx < cur_base + n) { it.c = c; it.q = cur_q; it.t = (int)(idx - cur_base); break; }
+                        cur_base += n;
+                        if (++cur_q == P) { cur_q = 0; ++cur_tau; }
+                    }
+                    // the phase before it must be complete for this matrix: its outputs are this item's operands, and the
+                    // buffers this item overwrites were last read two phases further back
+                    if (it.q > 0)
+                        ok = wait_counter(g.done + (size_t)it.c * P + (it.q - 1), 2u * (unsigned)g.ph[it.q - 1].items_per_mat, abort_flag, status, 6);
+                    fence_proxy_async();
+                    if (!ok) break;
+                }
+                const uint32_t slot = published % RING, par = (published / RING) & 1u;
+                if (!(ok = mbar_wait(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
+                asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
+                mbar_arrive_cluster(ring_full_own + 8 * slot);
+                mbar_arrive_cluster(ring_full_peer + 8 * slot);
+                ++published;
+                if (it.stop) break;
+                ok = produce(it);
+                idx = next_idx;
+            }
             // stay until the tensor cores have released every stage: the commits arrive on this CTA's barriers
+            for (int s = 0; s < STAGES && ok; ++s) {
+                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        } else if (lane == 0) {
+            // ---------------- TMA producer (peer) ----------------
+            bool ok = true;
+            for (unsigned n = 0; ok; ++n) {
+                Item it;
+                if (!(ok = take_item(n, it, 8, true)) || it.stop) break;
+                fence_proxy_async();       // the scheduler's acquire of the dependency precedes these copies
+                ok = produce(it);
+            }
             for (int s = 0; s < STAGES && ok; ++s) {
                 ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -373,20 +471,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
-            uint32_t stage = 0, phase = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
+            uint32_t mstage = 0, mphase = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
             bool ok = true;
-            for (int t = pair; t < total_tiles && ok; t += num_pairs) {
-                const TileCoord tc = decode_tile<WIDE>(g, t);
-                const bool shared_ab = !WIDE && g.ab_same && tc.tm == tc.tn;
-                const uint32_t acc0 = WIDE ? 0u : acc_next;
+            for (unsigned n = 0; ok; ++n) {
+                Item it;
+                if (!(ok = take_item(n, it, 9, true)) || it.stop) break;
+                const NsPhase& p = g.ph[it.q];
+                const TileCoord tc = decode_tile(p, it.t);
+                const bool shared_ab = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
+                const uint32_t acc0 = tc.nsub == 2 ? 0u : acc_next;
+                const int num_kb = (p.K + TC_BK - 1) / TC_BK;
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
-                    if (!(ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, status, 3))) break;
+                    if (!(ok = mbar_wait(bar_full + 8 * mstage, mphase, abort_flag, status, 3))) break;
                     tc_fence_after();
                     const int k0 = kb * TC_BK;
-                    const int a_mn = g.a_sym ? fetch_transposed(1, tc.tm, k0) : g.a_mn;
+                    const int a_mn = p.a_sym ? fetch_transposed(1, tc.tm, k0) : p.a_mn;
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
                     const uint32_t a_kstep = a_mn ? (2048u >> 4) : (32u >> 4);
-                    const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+                    const uint32_t sa = base + mstage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
                     const uint64_t da = smem_desc(sa, a_mn);
                     for (int u = 0; u < tc.nsub; ++u) {
                         const uint32_t acc = acc0 + u;
@@ -394,7 +496,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                             if (!(ok = mbar_wait(bar_acc_empty + 8 * acc, ((acc_par >> acc) & 1u) ^ 1u, abort_flag, status, 2))) break;
                             tc_fence_after();
                         }
-                        const int b_mn = shared_ab ? a_mn : (g.b_sym ? fetch_transposed(1, tc.tn + u, k0) : g.b_mn);
+                        const int b_mn = shared_ab ? a_mn : (p.b_sym ? fetch_transposed(1, tc.tn + u, k0) : p.b_mn);
                         const uint32_t b_kstep = b_mn ? (2048u >> 4) : (32u >> 4);
                         const uint64_t db = smem_desc(shared_ab ? sa : sb + u * B_SUB_BYTES, b_mn);
                         const uint32_t idesc = instr_desc(a_mn, b_mn);
@@ -405,8 +507,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                                         (kb | k) != 0 ? 1u : 0u);
                     }
                     if (!ok) break;
-                    tc_commit_pair(bar_empty + 8 * stage);     // frees the stage in both CTAs when these MMAs have read it
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    tc_commit_pair(bar_empty + 8 * mstage);     // frees the stage in both CTAs when these MMAs have read it
+                    if (++mstage == STAGES) { mstage = 0; mphase ^= 1u; }
                 }
                 if (!ok) break;
                 for (int u = 0; u < tc.nsub; ++u) {
@@ -414,107 +516,57 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                     tc_commit_pair(bar_acc_full + 8 * acc);    // accumulator complete, both CTAs' epilogues may read
                     acc_par ^= 1u << acc;
                 }
-                if (!WIDE) acc_next ^= 1u;
+                if (tc.nsub == 1) acc_next ^= 1u;
             }
         }
     } else {
         // ---------------- epilogue (warps 2..9, both CTAs) ----------------
         // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4).  A 256-column
-        // tile is written in phases of 128 columns; in a phase the two warps of a quadrant take 64 columns
-        // each, i.e. one 64 x 64 store box column.
+        // tile is handled in phases of 128 columns; in a phase the two warps of a quadrant take 64 columns
+        // each, so a thread owns 64 consecutive columns of one row: one 128-byte line of the bf16 output.
         const int quad = warp & 3;
         const int half = (warp - 2) >> 2;
         const int row_in_cta = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        const bool issuer = threadIdx.x == 64;                 // first epilogue thread: issues and retires TMA stores
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
-        // position of this thread's row inside the staging buffer: box (row half, column half), 128-byte rows
-        const uint32_t box_row = (uint32_t)(row_in_cta & 63);
-        const uint32_t stage_off = (uint32_t)(((row_in_cta >> 6) * 2 + half)) * BOX_BYTES + box_row * 128u;
-        const uint32_t swz = box_row & 7u;
-        uint32_t acc_next = 0, acc_par = 0, epi_it = 0;   // acc_par: one use-parity bit per accumulator
+        uint32_t acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
         bool alive = true;
-        for (int t = pair; t < total_tiles && alive; t += num_pairs) {
-            const TileCoord tc = decode_tile<WIDE>(g, t);
+        for (unsigned n = 0; alive; ++n) {
+            Item it;
+            bool got = take_item(n, it, 10, false);
+            got = epi_bar_all(3, got);         // all epilogue threads take the same exit, so no one is left at a barrier
+            if (!got) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(ring_empty_leader + 8 * (n % RING));   // every lane has its copy of the item
+            if (it.stop) break;
+            const NsPhase& p = g.ph[it.q];
+            const TileCoord tc = decode_tile(p, it.t);
             const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
             const int gr = m0 + row_in_cta;
-            const bool row_ok = gr < g.M;
-            const long long row_off = (long long)tc.c * g.mat_stride + (long long)gr * g.ld;
+            const bool row_ok = gr < p.M;
+            const long long row_off = (long long)it.c * p.mat_stride + (long long)gr * p.ld;
             float post = 1.0f;
-            if (g.post_mode) { const float sc = g.inv_norm[tc.c]; post = g.post_mode == 2 ? sc * sc : sc; }
-            const float c1 = g.c1 * post, c2 = g.c2 * post;
-            const uint32_t acc0 = WIDE ? 0u : acc_next;
-            for (int u = 0; u < tc.nsub; ++u) {
+            if (p.post_mode) { const float sc = g.inv_norm[it.c]; post = p.post_mode == 2 ? sc * sc : sc; }
+            const float c1 = p.c1 * post, c2 = p.c2 * post;
+            const uint32_t acc0 = tc.nsub == 2 ? 0u : acc_next;
+            for (int u = 0; u < tc.nsub && alive; ++u) {
                 const uint32_t acc = acc0 + u;
                 const int n0 = (tc.tn + u) * TC_BN;
-                const int nphases = (g.N - n0 > EPI_COLS) ? 2 : 1;
-                if constexpr (WIDE) {
-                    // Macro-tile configuration (no axpy operand, no diagonal term): both accumulators belong to the tile
-                    // in flight, so nothing hides this epilogue.  A thread's share of an accumulator (128 values) fits
-                    // in 64 packed registers: read and pack all of it first, hand the accumulator back to the MMA issuer,
-                    // and only then stage and store.
-                    bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
-                    ok = epi_bar_all(3, ok);
-                    if (!ok) { alive = false; break; }
-                    tc_fence_after();
-                    acc_par ^= 1u << acc;
-                    const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
-                    uint4 pk[2][8];
-                    #pragma unroll
-                    for (int ph = 0; ph < 2; ++ph) {
-                        if (ph < nphases) {
-                            float v[64];
-                            tmem_ld32(t_base + ph * EPI_COLS, v);
-                            tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
-                            tmem_ld_wait();
-                            #pragma unroll
-                            for (int j = 0; j < 64; ++j) v[j] *= c2;
-                            #pragma unroll
-                            for (int q = 0; q < 8; ++q) pk[ph][q] = pack8(v + 8 * q);
-                        }
-                    }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8 * acc);
-                    #pragma unroll
-                    for (int ph = 0; ph < 2; ++ph) {
-                        if (ph < nphases) {
-                            const uint32_t buf = epi_base + (epi_it % C::EPI_BUFS) * EPI_BUF_BYTES;
-                            if (issuer) bulk_wait_read<C::EPI_BUFS - 1>();
-                            epi_bar_sync(1);
-                            #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const uint32_t addr = buf + stage_off + (((uint32_t)q ^ swz) << 4);
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[ph][q].x), "r"(pk[ph][q].y),
-                                             "r"(pk[ph][q].z), "r"(pk[ph][q].w) : "memory");
-                            }
-                            fence_proxy_async();
-                            epi_bar_sync(2);
-                            if (issuer) {
-                                #pragma unroll
-                                for (int b = 0; b < 4; ++b) {
-                                    const int x = n0 + ph * EPI_COLS + (b & 1) * TC_BOX, y = m0 + (b >> 1) * TC_BOX;
-                                    if (x < g.N && y < g.M) tma_store_3d(&tma_d, buf + b * BOX_BYTES, x, y, tc.c);
-                                }
-                                bulk_commit();
-                            }
-                            ++epi_it;
-                        }
-                    }
-                } else {
-                // operand of the axpy term, requested before the accumulator is ready
+                const int nphases = (p.N - n0 > EPI_COLS) ? 2 : 1;
+                // operand of the axpy term, requested before the accumulator is ready.  It was written by other CTAs of this
+                // launch, so it is read from L2 (ld.cg), never from a line L1 may still hold from an earlier iteration.
                 uint4 cin_raw[8];
                 auto load_cin = [&](int ph) {
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
                     #pragma unroll
                     for (int q = 0; q < 8; ++q) {
-                        if (row_ok && gc0 + 8 * q < g.N) cin_raw[q] = *reinterpret_cast<const uint4*>(g.cin + row_off + gc0 + 8 * q);
+                        if (row_ok && gc0 + 8 * q < p.N) cin_raw[q] = __ldcg(reinterpret_cast<const uint4*>(p.cin + row_off + gc0 + 8 * q));
                         else cin_raw[q] = make_uint4(0u, 0u, 0u, 0u);
                     }
                 };
-                if (g.cin) load_cin(0);
+                if (p.cin) load_cin(0);
                 bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
-                ok = epi_bar_all(3, ok);           // all epilogue threads take the same exit, so no one is left at a barrier
+                ok = epi_bar_all(3, ok);
                 if (!ok) { alive = false; break; }
                 tc_fence_after();
                 acc_par ^= 1u << acc;
@@ -531,7 +583,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                         if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8 * acc);
                     }
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
-                    if (g.cin) {
+                    if (p.cin) {
                         const uint32_t w[32] = {cin_raw[0].x, cin_raw[0].y, cin_raw[0].z, cin_raw[0].w, cin_raw[1].x, cin_raw[1].y,
                                                 cin_raw[1].z, cin_raw[1].w, cin_raw[2].x, cin_raw[2].y, cin_raw[2].z, cin_raw[2].w,
                                                 cin_raw[3].x, cin_raw[3].y, cin_raw[3].z, cin_raw[3].w, cin_raw[4].x, cin_raw[4].y,
@@ -548,38 +600,45 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
                         #pragma unroll
                         for (int j = 0; j < 64; ++j) v[j] *= c2;
                     }
-                    if (g.diag_add != 0.f && gr >= gc0 && gr < gc0 + 64) {
+                    if (p.diag_add != 0.f && gr >= gc0 && gr < gc0 + 64) {
                         #pragma unroll
-                        for (int j = 0; j < 64; ++j) v[j] += (gc0 + j == gr) ? g.diag_add : 0.f;
+                        for (int j = 0; j < 64; ++j) v[j] += (gc0 + j == gr) ? p.diag_add : 0.f;
                     }
-                    // the staging buffer is free once the stores issued EPI_BUFS phases ago have read it
-                    const uint32_t buf = epi_base + (epi_it % C::EPI_BUFS) * EPI_BUF_BYTES;
-                    if (issuer) bulk_wait_read<C::EPI_BUFS - 1>();
-                    epi_bar_sync(1);
-                    #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const uint4 pk = pack8(v + 8 * q);
-                        const uint32_t addr = buf + stage_off + (((uint32_t)q ^ swz) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk.x), "r"(pk.y), "r"(pk.z), "r"(pk.w)
-                                     : "memory");
-                    }
-                    fence_proxy_async();           // generic-proxy writes above must be visible to the TMA engine
-                    epi_bar_sync(2);
-                    if (issuer) {
+                    if (!row_ok) continue;
+                    if (!p.fuse_update) {
+                        __nv_bfloat16* drow = p.d + row_off + gc0;
                         #pragma unroll
-                        for (int b = 0; b < 4; ++b) {
-                            const int x = n0 + ph * EPI_COLS + (b & 1) * TC_BOX, y = m0 + (b >> 1) * TC_BOX;
-                            if (x < g.N && y < g.M) tma_store_3d(&tma_d, buf + b * BOX_BYTES, x, y, tc.c);   // clipped at the extents
-                        }
-                        bulk_commit();
-                    }
-                    ++epi_it;
-                }
+                        for (int q = 0; q < 8; ++q)
+                            if (gc0 + 8 * q < p.N) *reinterpret_cast<uint4*>(drow + 8 * q) = pack8(v + 8 * q);
+                    } else {
+                        // Eq. muon_update on this thread's 64 parameters: W <- (W - eta lambda W) - eta gamma O
+                        float* wrow = upd.w[it.c] + (long long)gr * p.ld + gc0;
+                        float* orow = upd.o[it.c] ? upd.o[it.c] + (long long)gr * p.ld + gc0 : nullptr;
+                        #pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            if (gc0 + 8 * q < p.N) {
+                                float w8[8];
+                                ld8(wrow + 8 * q, w8);
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j) w8[j] = fmaf(-g.eta_gamma, v[8 * q + j], fmaf(-g.eta_lambda, w8[j], w8[j]));
+                                st8(wrow + 8 * q, w8);
+                                if (orow) st8(orow + 8 * q, v + 8 * q);
                             }
-}
-            if (!WIDE) acc_next ^= 1u;
+                        }
+                    }
+                }
+            }
+            if (!alive) break;
+            if (tc.nsub == 1) acc_next ^= 1u;
+            // count the item as done for its matrix and phase: every thread's stores, fenced, then one arrival per CTA
+            fence_proxy_async();
+            __threadfence();
+            epi_bar_sync(1);
+            if (threadIdx.x == 64) {
+                __threadfence();
+                atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
+            }
         }
-        if (issuer) bulk_wait_all();           // shared memory must outlive the stores that read it
     }
 
     if (*abort_flag) __nanosleep(200000);      // let copies that are still in flight land before the CTA goes away
@@ -595,59 +654,60 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tma_a, const __grid_constant_
 
 }  // namespace
 
-void tc_gemm_plan(TcGemm& g) {
-    g.tiles_m = (g.M + TC_BM - 1) / TC_BM;
-    g.tiles_n = (g.N + TC_BN - 1) / TC_BN;
-    if (g.symmetric) g.wide = 0;
-    if (g.wide) g.tiles_per_mat = g.tiles_m * ((g.tiles_n + 1) / 2);
-    else g.tiles_per_mat = g.symmetric ? g.tiles_m * (g.tiles_m + 1) / 2 : g.tiles_m * g.tiles_n;
+void ns_phase_plan(NsPhase& p) {
+    p.tiles_m = (p.M + TC_BM - 1) / TC_BM;
+    p.tiles_n = (p.N + TC_BN - 1) / TC_BN;
+    if (p.symmetric || p.tiles_n < 2) p.wide = 0;      // a macro-tile needs two tile columns to pay
+    if (p.wide) p.items_per_mat = p.tiles_m * ((p.tiles_n + 1) / 2);
+    else p.items_per_mat = p.symmetric ? p.tiles_m * (p.tiles_m + 1) / 2 : p.tiles_m * p.tiles_n;
 }
 
-double tc_gemm_executed_flops(const TcGemm& g) {
-    const double kpad = (double)((g.K + TC_BK - 1) / TC_BK * TC_BK);
-    const double tiles256 = g.symmetric ? g.tiles_m * (g.tiles_m + 1) / 2 : g.tiles_m * g.tiles_n;
-    return 2.0 * TC_BM * TC_BN * kpad * tiles256 * g.C;
+double ns_phase_executed_flops(const NsPhase& p) {
+    const double kpad = (double)((p.K + TC_BK - 1) / TC_BK * TC_BK);
+    const double tiles256 = p.symmetric ? p.tiles_m * (p.tiles_m + 1) / 2 : p.tiles_m * p.tiles_n;
+    return 2.0 * TC_BM * TC_BN * kpad * tiles256;
 }
 
-namespace {
-template <bool WIDE>
-cudaError_t configure_one(int sms, int* clusters) {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel<WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<WIDE>::SMEM_TOTAL);
-    if (e != cudaSuccess) return e;
+void ns_program_plan(NsProgram& g) {
+    unsigned long long total = 0;
+    for (int q = 0; q < g.P; ++q) total += (unsigned long long)g.ph[q].items_per_mat * (unsigned long long)g.C;
+    g.total_items = (unsigned int)total;
+}
+
+cudaError_t ns_configure(int* max_pairs) {
+    int dev = 0, sms = 0;
+    cudaError_t e;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(ns_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_TOTAL)) != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(sms / 2 * 2));
     cfg.blockDim = dim3(TC_THREADS);
-    cfg.dynamicSmemBytes = Cfg<WIDE>::SMEM_TOTAL;
+    cfg.dynamicSmemBytes = SMEM_TOTAL;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    return cudaOccupancyMaxActiveClusters(clusters, tc_gemm_kernel<WIDE>, &cfg);
-}
-}  // namespace
-
-cudaError_t tc_gemm_configure(int* max_pairs) {
-    int dev = 0, sms = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    int c0 = 0, c1 = 0;
-    if ((e = configure_one<false>(sms, &c0)) != cudaSuccess) return e;
-    if ((e = configure_one<true>(sms, &c1)) != cudaSuccess) return e;
-    const int clusters = c0 < c1 ? c0 : c1;
+    int clusters = 0;
+    if ((e = cudaOccupancyMaxActiveClusters(&clusters, ns_chunk_kernel, &cfg)) != cudaSuccess) return e;
     if (clusters < 1) return cudaErrorInvalidConfiguration;
     *max_pairs = clusters < sms / 2 ? clusters : sms / 2;
     return cudaSuccess;
 }
 
-cudaError_t launch_tc_gemm(const CUtensorMap& tma_a, const CUtensorMap& tma_b, const CUtensorMap& tma_d,
-                           const TcGemm& g, int max_pairs, DeviceStatus* status, cudaStream_t stream) {
-    const int total = g.C * g.tiles_per_mat;
-    if (total <= 0) return cudaSuccess;
-    const int pairs = total < max_pairs ? total : max_pairs;
-    if (g.wide) tc_gemm_kernel<true><<<2 * pairs, TC_THREADS, Cfg<true>::SMEM_TOTAL, stream>>>(tma_a, tma_b, tma_d, g, status);
-    else        tc_gemm_kernel<false><<<2 * pairs, TC_THREADS, Cfg<false>::SMEM_TOTAL, stream>>>(tma_a, tma_b, tma_d, g, status);
+cudaError_t launch_ns_program(const NsMaps& maps, const NsProgram& g, const NsUpdatePtrs& up, int max_pairs,
+                              DeviceStatus* status, cudaStream_t stream) {
+    if (g.total_items == 0) return cudaSuccess;
+    const int pairs = (long long)g.total_items < (long long)max_pairs ? (int)g.total_items : max_pairs;
+    static const UpdateTable no_update = {};
+    const UpdateTable* table = &no_update;
+    UpdateTable filled;
+    if (up.w) {
+        for (int c = 0; c < g.C; ++c) { filled.w[c] = up.w[c]; filled.o[c] = up.o ? up.o[c] : nullptr; }
+        table = &filled;
+    }
+    ns_chunk_kernel<<<2 * pairs, TC_THREADS, SMEM_TOTAL, stream>>>(maps, g, *table, status);
     return cudaGetLastError();
 }
 

@@ -1,5 +1,6 @@
-// Tensor-core Newton-Schulz GEMMs (definitions in ns_tc.cu): tcgen05.mma issued for a pair of CTAs
-// (cta_group::2), TMA-staged bf16 tiles, fp32 accumulators in tensor memory, TMA-store epilogue.
+// Tensor-core Newton-Schulz iteration (definitions in ns_tc.cu): one persistent kernel per chunk runs all
+// GEMMs of up to five iterations of Eq. newton_schulz.  tcgen05.mma is issued for a pair of CTAs
+// (cta_group::2), operands are TMA-staged bf16 tiles, accumulators are fp32 in tensor memory.
 #pragma once
 #include <cuda.h>
 
@@ -11,49 +12,88 @@ constexpr int TC_BM = 256;      // rows of D per tile: one CTA pair, 128 rows pe
 constexpr int TC_BN = 256;      // columns of D per tile (UMMA N = 256, each CTA stages 128 of them)
 constexpr int TC_BK = 64;       // k-slice per pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_BOX = 64;      // every TMA box is 64 (contiguous) x 64 (strided) bf16 = 8 KiB
+constexpr int NS_MAX_PHASES = 15;   // 3 GEMMs x 5 iterations per launch; longer iterations take several launches
+constexpr int NS_MAPS = 4;          // operand tensors of a chunk: X ping, X pong, A, B'
 
-// One batched GEMM of the iteration of Eq. newton_schulz over the C matrices of a chunk:
+// One batched GEMM ("phase") of the iteration of Eq. newton_schulz over the C matrices of a chunk:
 //     D = post * (c1 * Cin + c2 * Aop x Bop^T) + diag_add * I,   D, Cin bf16; accumulation fp32.
-// Operand tiles and the output go through tensor maps over [C][rows][cols] bf16 tensors.  An operand
-// is "K-major" when k is its contiguous index and "MN-major" when its row index is contiguous; tall
-// weights use the MN-major form so that X^T X and B X need no transposed copy.
+// Operand tiles are fetched through tensor maps over [C][rows][cols] bf16 tensors; D and Cin are addressed
+// directly.  An operand is "K-major" when k is its contiguous index and "MN-major" when its row index is
+// contiguous; tall weights use the MN-major form so that X^T X and X B' need no transposed copy.
 //
 // Symmetric matrices (X X^T, b A + c A^2 + a I) are only ever stored in their lower block triangle:
 // with `symmetric` set, only the 256 x 256 tiles with tile row >= tile column are computed and
 // written (diagonal tiles completely).  A consumer that needs a block above the diagonal fetches the
 // stored block below it as an MN-major operand instead (`a_sym` / `b_sym`), so nothing is mirrored.
-struct TcGemm {
-    int C;                      // matrices in the launch
+//
+// With `fuse_update` set (the last X' = B' X of a step) D is not stored: the epilogue applies
+// Eq. muon_update, W <- (W - eta lambda W) - eta gamma D, to the fp32 parameter of the same matrix
+// straight from the fp32 accumulator, and writes D itself (fp32) only where an output pointer is given.
+struct NsPhase {
     int M, N, K;                // per-matrix GEMM extents
+    int a_map, b_map;           // which of the chunk's tensor maps the operands come from
     int a_mn, b_mn;             // 1: operand is MN-major (ignored for an operand flagged *_sym)
     int a_sym, b_sym;           // 1: operand is a symmetric matrix stored as its lower block triangle
     int symmetric;              // 1: D = D^T, compute lower-triangle tiles only
     int ab_same;                // 1: both operands are the same tensor in the same form (X X^T, A A): a diagonal
                                 //    tile stages its operand rows once and uses them on both sides
-    int wide;                   // 1 (non-symmetric D only): a pair computes 256 x 512 macro-tiles, two tiles that share
+    int wide;                   // 1 (non-symmetric D only): a work item is a 256 x 512 macro-tile, two tiles that share
                                 //    one staged slice of the A operand, one per tensor-memory accumulator
-    int tiles_m, tiles_n, tiles_per_mat;   // tiles_per_mat counts macro-tiles when `wide`
-    const __nv_bfloat16* cin;   // may be null; when D is symmetric, Cin is lower-block-stored like D
-    long long ld, mat_stride;   // leading dimension and per-matrix stride of cin, in elements
+    int tiles_m, tiles_n, items_per_mat;   // filled by ns_phase_plan(); items are macro-tiles when `wide`
+    __nv_bfloat16* d;           // output [C][M][N] (dense), unused when fuse_update
+    const __nv_bfloat16* cin;   // may be null; same layout as d; lower-block-stored when D is symmetric
+    long long ld, mat_stride;   // leading dimension and per-matrix stride of d and cin, in elements
     float c1, c2;
     float diag_add;             // added to D(i,i): folds the a*X term of the quintic into B' = b A + c A^2 + a I
+    int post_mode;              // 0: post = 1, 1: post = inv_norm[c], 2: post = inv_norm[c]^2
+    int fuse_update;            // 1: epilogue applies the parameter update instead of storing D
+};
+
+// Everything one launch needs: the phases in execution order and the scheduler state.  Work items are handed
+// out through one atomic counter in a fixed order in which every item comes after the items it depends on
+// (phase q of matrix c follows phase q - 1 of matrix c by `delay` matrices), so a pair that has taken an item
+// only ever waits for items already taken by running pairs; completion of a phase of a matrix is counted in
+// done[c * P + q] (two arrivals per item, one from each CTA of the pair).
+struct NsProgram {
+    int C;                      // matrices in the chunk
+    int P;                      // phases in this launch (<= NS_MAX_PHASES)
+    int delay;                  // distance, in matrices, between consecutive phases of one matrix in the item order
+    unsigned int total_items;
+    NsPhase ph[NS_MAX_PHASES];
     const float* inv_norm;      // per-matrix 1/(||M||_F + eps), used when post_mode != 0
-    int post_mode;              // 0: post = 1, 1: post = inv, 2: post = inv^2
+    unsigned int* work_counter; // zero at launch
+    unsigned int* done;         // C * P words, zero at launch
+    float eta_lambda, eta_gamma;    // fuse_update: eta * lambda and eta * gamma
     int selftest_extra_tx;      // 0 in normal use.  The time-out self-test sets it: every stage then expects this many
                                 //    bytes more than its copies deliver, so the "full" wait runs out and the kernel must
                                 //    report STATUS_TIMEOUT and leave cleanly (all copies still complete; nothing faults)
 };
 
-// Fills the tile counts of `g` from M, N, symmetric, wide.
-void tc_gemm_plan(TcGemm& g);
-// Tensor-core flops (2*M*N*K per issued MMA, padded extents included) one launch of `g` executes.
-double tc_gemm_executed_flops(const TcGemm& g);
+struct alignas(64) NsMaps {
+    CUtensorMap m[NS_MAPS];
+};
+
+// Per-matrix parameter and optional fp32 output pointers for a phase with fuse_update: HOST arrays of C device
+// pointers (copied into the launch's arguments).  w == nullptr: no phase of the launch fuses the update.
+struct NsUpdatePtrs {
+    float* const* w;
+    float* const* o;            // entries may be null; the array itself may be null
+};
+
+// Fills the tile counts of `p` from M, N, symmetric, wide.
+void ns_phase_plan(NsPhase& p);
+// Tensor-core flops one matrix costs in phase `p`: executed (2*M*N*K per issued 256 x 256 tile MMA, padded
+// extents and the upper halves of diagonal tiles included).
+double ns_phase_executed_flops(const NsPhase& p);
+// Fills total_items from C, P, the phases' item counts.
+void ns_program_plan(NsProgram& g);
+// Words of scheduler scratch (work counter + done counters) a launch over C matrices and P phases needs zeroed.
+inline size_t ns_sched_words(int C, int P) { return 64 + (size_t)C * P; }
 
 // Sets the kernel's shared-memory attribute and finds how many CTA pairs the device holds at once.
 // Call once per device before the first launch.
-cudaError_t tc_gemm_configure(int* max_pairs);
-// tma_a / tma_b: operand tensors, tma_d: output tensor (all bf16, 64 x 64 boxes, 128-byte swizzle).
-cudaError_t launch_tc_gemm(const CUtensorMap& tma_a, const CUtensorMap& tma_b, const CUtensorMap& tma_d,
-                           const TcGemm& g, int max_pairs, DeviceStatus* status, cudaStream_t stream);
+cudaError_t ns_configure(int* max_pairs);
+cudaError_t launch_ns_program(const NsMaps& maps, const NsProgram& g, const NsUpdatePtrs& upd, int max_pairs,
+                              DeviceStatus* status, cudaStream_t stream);
 
 }  // namespace mona

@@ -7,7 +7,7 @@ import pytest
 
 import paper_2605_26842_b200 as pkg
 from paper_2605_26842_b200 import synth
-from tests.parity_util import TOL_O_BF16, TOL_STATE, TOL_W, run_case
+from tests.parity_util import TOL_O_BF16, TOL_O_MAX_BF16, TOL_STATE, TOL_STATE_MAX, TOL_W, run_case
 
 pytestmark = pytest.mark.gpu
 
@@ -25,8 +25,21 @@ def test_one_layer_of_the_7b_set_sampled():
     assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE and errs["Gprev"] <= TOL_STATE, errs
     assert errs["O"] <= TOL_O_BF16 and errs["dW"] <= TOL_W, errs
     # buckets: 128 wide experts (2 chunks), 64 tall experts, 4 attention matrices, 1 shared expert: 5 chunks,
-    # each one prologue + 15 GEMMs + one update
-    assert errs["launches"] == 5 * 17, errs["launches"]
+    # each one prologue + one Newton-Schulz launch (all 15 GEMMs, the update in the last one's epilogue)
+    assert errs["launches"] == 5 * 2, errs["launches"]
+
+
+def test_one_layer_of_the_7b_set_ten_steps():
+    """The "parameters after 10 steps" clause at benchmark scale: the same one-layer set, ten steps, a sample of
+    matrices from every bucket followed by the oracle throughout and compared after step 10."""
+    wl = synth.workload(3, layers=1)
+    shapes = [(s.batch, s.rows, s.cols) for s in wl.specs]
+    sample = {0: [37], 1: [28, 29], 2: [63], 3: [0], 7: [0]}
+    hp = pkg.default_hparams(accel_beta=wl.accel_beta, accel_alpha=wl.accel_alpha)
+    errs = run_case(shapes, steps=10, hp=hp, rho=wl.rho, sigma=wl.sigma, seed=wl.seed + 1, sample=sample, heavy_tail=True, check_at={10})
+    assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE and errs["Gprev"] <= TOL_STATE, errs
+    assert errs["M_max"] <= TOL_STATE_MAX and errs["A_max"] <= TOL_STATE_MAX, errs
+    assert errs["O"] <= TOL_O_BF16 and errs["O_max"] <= TOL_O_MAX_BF16 and errs["dW"] <= TOL_W, errs
 
 
 def test_shard_stress_shapes_with_bf16_gradients():

@@ -3,8 +3,8 @@ import pytest
 import torch
 
 import paper_2605_26842_b200 as pkg
-from tests.parity_util import (LITE_MAX_FLIPPED, TOL_A_LITE, TOL_M_LITE, TOL_O_BF16, TOL_O_FP32, TOL_STATE, TOL_W,
-                               run_case)
+from tests.parity_util import (LITE_MAX_FLIPPED, TOL_A_LITE, TOL_M_LITE, TOL_O_BF16, TOL_O_FP32, TOL_O_MAX_BF16,
+                               TOL_O_MAX_FP32, TOL_STATE, TOL_STATE_MAX, TOL_W, run_case)
 
 pytestmark = pytest.mark.gpu
 
@@ -13,6 +13,9 @@ def check(errs, tol_o):
     assert errs["M"] <= TOL_STATE and errs["A"] <= TOL_STATE and errs["Gprev"] <= TOL_STATE, errs
     assert errs["O"] <= tol_o, errs
     assert errs["dW"] <= max(TOL_W, tol_o), errs
+    # no single element far off (an unwritten or misplaced patch would pass the Frobenius gates)
+    assert errs["M_max"] <= TOL_STATE_MAX and errs["A_max"] <= TOL_STATE_MAX and errs["Gprev_max"] <= TOL_STATE_MAX, errs
+    assert errs["O_max"] <= (TOL_O_MAX_FP32 if tol_o == TOL_O_FP32 else TOL_O_MAX_BF16), errs
 
 
 def test_config0_fp32_validation():
@@ -58,6 +61,73 @@ def test_mixed_set_ten_steps():
     shapes = [(4, 256, 512), (4, 512, 256), (1, 512, 512), (1, 32, 512)]
     errs = run_case(shapes, steps=10, seed=42)
     check(errs, TOL_O_BF16)
+
+
+def test_separate_update_kernel_matches_too():
+    """fuse_update = 0: O_k stored in bf16 and a separate elementwise kernel applies Eq. muon_update."""
+    shapes = [(3, 256, 512), (2, 512, 256), (1, 320, 192)]
+    errs = run_case(shapes, steps=3, seed=43, options=pkg.default_options(fuse_update=0))
+    check(errs, TOL_O_BF16)
+    assert errs["launches"] == 3 * 3        # per chunk: prologue, Newton-Schulz, update
+
+
+@pytest.mark.parametrize("delay", [1, 2, 7])
+def test_work_order_delay_does_not_change_results(delay):
+    """ns_delay only moves work items in the kernel's hand-out order: results are bit-identical to the default."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(19)
+    shapes = [(9, 256, 384), (3, 512, 256)]
+    W0 = [torch.randn(s, generator=gen) * 0.02 for s in shapes]
+    G = [[torch.randn(s, generator=gen) * 1e-3 for s in shapes] for _ in range(2)]
+    hp = pkg.default_hparams()
+
+    def run(opts):
+        p = [w.clone().to(dev) for w in W0]
+        opt = pkg.MonaOptimizer(p, options=opts)
+        for k in range(2):
+            opt.step(hp, p, [g.to(dev) for g in G[k]])
+        torch.cuda.synchronize()
+        assert opt.poll_status()[0] == 0
+        out = [t.clone() for t in p]
+        opt.close()
+        return out
+    a, b = run(pkg.default_options()), run(pkg.default_options(ns_delay=delay))
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def test_zero_gradient_from_zero_state():
+    """M = 0 (zero gradient, zero state): X_0 = 0 / (0 + eps) = 0, so O_k is exactly 0, only weight decay acts,
+    W <- (1 - eta lambda) W, and nothing is reported (the norm is finite).  Both Newton-Schulz paths."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(2)
+    shapes = [(2, 256, 384), (1, 384, 256), (1, 32, 256), (1, 33, 17)]
+    for precision in (0, 1):
+        hp = pkg.default_hparams(ns_precision=precision)
+        p = [(torch.randn(s, generator=gen) * 0.02).to(dev) for s in shapes]
+        w0 = [t.clone() for t in p]
+        g = [torch.zeros(s, device=dev) for s in shapes]
+        o = [torch.full(s, 7.0, device=dev) for s in shapes]
+        opt = pkg.MonaOptimizer(p)
+        opt.step_ex(hp, p, g, o, 7)
+        st, bad = opt.poll_status()
+        assert st == 0 and bad == -1
+        for i in range(len(shapes)):
+            assert torch.count_nonzero(o[i]).item() == 0
+            for view in opt.state_views(i):
+                assert torch.count_nonzero(view).item() == 0
+            expect = w0[i].double() * (1.0 - hp.lr * hp.weight_decay)
+            assert (p[i].double() - expect).abs().max().item() <= 1e-7 * w0[i].abs().max().item()
+        opt.close()
+
+
+def test_alpha_zero_is_muon():
+    """alpha = 0: Algorithm 1 with the acceleration weight switched off must take Muon's steps (M, O, W against the
+    oracle's separately written Muon), although A and G_prev still evolve."""
+    hp = pkg.default_hparams(accel_alpha=0.0)
+    errs = run_case([(2, 256, 384), (1, 384, 128), (1, 40, 72)], steps=4, hp=hp, seed=29, muon=True, compare_aux=False)
+    assert errs["M"] <= TOL_STATE and errs["M_max"] <= TOL_STATE_MAX, errs
+    assert errs["O"] <= TOL_O_BF16 and errs["O_max"] <= TOL_O_MAX_BF16 and errs["dW"] <= TOL_W, errs
 
 
 def test_bf16_gradients_and_padding():
