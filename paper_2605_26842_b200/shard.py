@@ -5,8 +5,12 @@ Every matrix's update is independent of every other matrix (Algorithm 1 is writt
 step shards by whole matrices with no data-path collective.  Two uses:
 
   * weak scaling (the benchmark): every rank owns a full parameter set of the same shape;
-  * a ZeRO-1-style deployment: one parameter set is split across ranks with `partition()`, each rank runs
-    its own handle over its share, and the updated weights are exchanged afterwards by the framework.
+  * a ZeRO-1-style deployment (the distributed Muon scheme the paper's related-work section cites): one
+    parameter set is split across ranks with `partition()`, each rank steps the matrices it owns
+    (`local_views()` gives the slices of the full tensors, which is what a handle is built over), and
+    `exchange()` then brings every rank's copy of the parameters up to date - one broadcast per owned slice,
+    in place, no staging copy.  That exchange is the only collective; it follows the step, it is not fused
+    with it (there is no computation left to overlap it with).
 """
 from __future__ import annotations
 
@@ -64,6 +68,38 @@ def partition(shapes: Sequence[Tuple[int, int, int]], world: int, ns_steps: int 
 
 def loads(shapes: Sequence[Tuple[int, int, int]], shares: List[List[Share]], ns_steps: int = 5) -> List[float]:
     return [sum(sh.count * step_cost(shapes[sh.spec][1], shapes[sh.spec][2], ns_steps) for sh in rank) for rank in shares]
+
+
+def local_views(tensors, shares: Sequence[Share]):
+    """The slices of the full per-descriptor tensors (batch, rows, cols) that `shares` names, as views:
+    stepping them steps the owner's part of the full parameter set in place."""
+    return [tensors[sh.spec][sh.start: sh.start + sh.count] for sh in shares]
+
+
+def share_shapes(shapes: Sequence[Tuple[int, int, int]], shares: Sequence[Share]) -> List[Tuple[int, int, int]]:
+    """(count, rows, cols) of every share: the descriptor list of the owner's handle."""
+    return [(sh.count, shapes[sh.spec][1], shapes[sh.spec][2]) for sh in shares]
+
+
+def exchange(params, all_shares: List[List[Share]], dist=None) -> int:
+    """After every rank has stepped the matrices it owns: make all ranks' full parameter tensors equal by
+    broadcasting each owned slice from its owner, in place.  `params` are this rank's full tensors
+    (batch, rows, cols).  Returns the bytes this rank received.  With dist=None (one process) there is nothing
+    to do.  Slices are contiguous (stacked descriptors are cut along the batch axis), so no packing is needed;
+    the broadcasts are issued asynchronously and waited for together."""
+    if dist is None or len(all_shares) == 1:
+        return 0
+    me = dist.get_rank()
+    works, received = [], 0
+    for owner, lst in enumerate(all_shares):
+        for sh in lst:
+            view = params[sh.spec][sh.start: sh.start + sh.count]
+            works.append(dist.broadcast(view, src=owner, async_op=True))
+            if owner != me:
+                received += view.numel() * view.element_size()
+    for w in works:
+        w.wait()
+    return received
 
 
 def env_rank() -> Tuple[int, int, int]:
