@@ -127,7 +127,8 @@ mona_status mona_default_hparams(mona_hparams* hp);
  *                        re-read, no separate update kernel).  0: O_k is stored in bf16 and a separate elementwise
  *                        kernel updates the parameters.  The two differ by the bf16 rounding of O_k only.
  *   ns_delay           : how many matrices apart consecutive Newton-Schulz GEMMs of one matrix sit in the kernel's
- *                        work order (0 = the default, 3; at most 64).  Larger values hide the dependency latency
+ *                        work order (0 = the default, 3; at most 1024; a value >= the chunk's matrix count
+ *                        runs the chunk GEMM by GEMM).  Larger values hide the dependency latency
  *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it. */
 typedef struct {
     size_t chunk_budget_bytes;

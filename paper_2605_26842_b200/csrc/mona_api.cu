@@ -2,6 +2,7 @@
 // and the per-step launch sequence.  See include/mona.h for the contract of every entry point.
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <atomic>
@@ -53,6 +54,14 @@ std::atomic<int> g_chunk_overlap{1};
 std::atomic<size_t> g_chunk_budget_bytes{DEFAULT_CHUNK_BUDGET};
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// NVTX range over the host-side enqueue of a phase (shows up in timeline tools; costs nothing without one attached).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 struct MatRef {
     int desc;
@@ -260,7 +269,7 @@ mona_status resolve_options(const mona_options* in, mona_options& out) {
     }
     out.chunk_overlap = in->chunk_overlap ? 1 : 0;
     out.fuse_update = in->fuse_update ? 1 : 0;
-    if (in->ns_delay < 0 || in->ns_delay > 64) return MONA_ERR_INVALID_ARG;
+    if (in->ns_delay < 0 || in->ns_delay > 1024) return MONA_ERR_INVALID_ARG;
     if (in->ns_delay > 0) out.ns_delay = in->ns_delay;
     return MONA_OK;
 }
@@ -297,7 +306,7 @@ mona_status mona_create_opt(mona_handle** out, const mona_matrix_desc* descs, in
     mona_handle* h = new mona_handle();
     *out = h;     // returned even on failure so that mona_last_error() can be read; destroy it either way
     if (resolve_options(options, h->opt) != MONA_OK)
-        return h->fail(MONA_ERR_INVALID_ARG, "options: chunk_budget_bytes must be 0 or at least 1 MiB, ns_delay within 0..64");
+        return h->fail(MONA_ERR_INVALID_ARG, "options: chunk_budget_bytes must be 0 or at least 1 MiB, ns_delay within 0..1024");
     mona_status st = build_plan(descs, n_desc, h->opt.chunk_budget_bytes, h->plan, h->last_error);
     if (st != MONA_OK) return st;
     if (!state || !workspace) return h->fail(MONA_ERR_INVALID_ARG, "state or workspace is null");
@@ -367,6 +376,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
             return h->fail(MONA_ERR_ALIGNMENT, "descriptor %lld: pointers must be 16-byte aligned", (long long)i);
     }
     MONA_CUDA(h, cudaSetDevice(h->device));
+    NvtxRange step_range("mona_step");
 
     PrologueScalars ps;
     ps.beta = split(hp->accel_beta);
@@ -445,6 +455,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
             if (params_host)
                 for (int dsc : chunk_descs) MONA_CUDA(h, cudaStreamWaitEvent(stream, h->ev_in[dsc], 0));
             if (phase_mask & 1u) {
+                NvtxRange range("mona.prologue");
                 MONA_CUDA(h, launch_prologue(ptrs, C, b.grad_dtype == MONA_BF16,
                                              hp->algorithm == 1 ? PROLOGUE_NO_AUX : (b.state_dtype == MONA_BF16 ? PROLOGUE_AUX_BF16 :
                                                  b.state_dtype == MONA_STATE_COMBINED ? PROLOGUE_AUX_COMBINED : PROLOGUE_AUX_F32), vec4, Mc, Ac, Gc, tc ? xb[0] : nullptr, partials,
@@ -455,13 +466,13 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
             bool update_fused = false;
             if (tc) {
                 if (phase_mask & 2u) {
+                    NvtxRange range("mona.newton_schulz");
                     // the last X' = B' X applies the parameter update in its epilogue when this call runs both phases and the
                     // fp32 rows can be accessed 32 bytes at a time
                     update_fused = h->opt.fuse_update && (phase_mask & 4u) != 0u;
                     for (int c = 0; c < C && update_fused; ++c)
                         if (((uintptr_t)ptrs.w[c] & 31) || ((uintptr_t)ptrs.o[c] & 31)) update_fused = false;
                     unsigned int* sched = (unsigned int*)(ctrl + CTRL_SCHED_OFF);
-                    __nv_bfloat16* bb = (__nv_bfloat16*)(data + b.off_b);
                     for (int t0 = 0; t0 < T; t0 += NS_MAX_PHASES / 3) {
                         const int t1 = std::min(T, t0 + NS_MAX_PHASES / 3);
                         NsProgram g{};
@@ -472,15 +483,15 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                             const int cur = t & 1, nxt = cur ^ 1;
                             NsPhase& g1 = g.ph[3 * (t - t0)];      // A = X X^T (wide) or X^T X (tall): lower-triangle tiles only
                             g1.M = g1.N = (int)b.s; g1.K = (int)b.l; g1.a_map = g1.b_map = MAP_X0 + cur; g1.a_mn = g1.b_mn = b.tall ? 1 : 0;
-                            g1.symmetric = 1; g1.ab_same = 1; g1.d = ab; g1.ld = b.s; g1.mat_stride = b.s * b.s;
+                            g1.symmetric = 1; g1.ab_same = 1; g1.d_map = MAP_A; g1.ld = b.s; g1.mat_stride = b.s * b.s;
                             g1.c1 = 0.f; g1.c2 = 1.f; g1.post_mode = t == 0 ? 2 : 0;
                             ns_phase_plan(g1);
                             NsPhase& g2 = g.ph[3 * (t - t0) + 1];  // B' = b A + c A A + a I, operands and result lower-block-stored
                             g2.M = g2.N = g2.K = (int)b.s; g2.a_map = g2.b_map = MAP_A; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
-                            g2.cin = ab; g2.d = bb; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c; g2.diag_add = ns_a;
+                            g2.cin = ab; g2.d_map = MAP_B; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c; g2.diag_add = ns_a;
                             ns_phase_plan(g2);
                             NsPhase& g3 = g.ph[3 * (t - t0) + 2];  // X' = B' X (wide) or X B' (tall), 256 x 512 macro-tiles
-                            g3.K = (int)b.s; g3.wide = 1; g3.d = xb[nxt]; g3.ld = b.cols; g3.mat_stride = b.e;
+                            g3.K = (int)b.s; g3.wide = 1; g3.d_map = MAP_X0 + nxt; g3.ld = b.cols; g3.mat_stride = b.e;
                             g3.c1 = 0.f; g3.c2 = 1.f; g3.post_mode = t == 0 ? 1 : 0;
                             g3.fuse_update = (update_fused && t == T - 1) ? 1 : 0;
                             if (!b.tall) {   // B' is the symmetric "A" operand, X the MN-major "B" operand
@@ -505,6 +516,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
             } else if (small_ns_eligible(b.rows, b.cols)) {
                 // short side <= 64 (routers): the whole iteration in one launch, one block per matrix
                 if (phase_mask & 2u) {
+                    NvtxRange range("mona.newton_schulz.small");
                     MONA_CUDA(h, launch_small_ns(Mc, xf[0], inv_norm, C, (int)b.rows, (int)b.cols, T, ns_a, ns_b, ns_c, stream));
                     ++h->launches;
                     h->flops_dense += (double)T * C * (4.0 * b.s * b.s * b.l + 2.0 * (double)b.s * b.s * b.s);
@@ -512,6 +524,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                 o_final = xf[0];
             } else {
                 if (phase_mask & 2u) {
+                    NvtxRange range("mona.newton_schulz.fp32");
                     MONA_CUDA(h, launch_scale(Mc, xf[0], inv_norm, C, b.e, b.slab_len, b.slabs, stream));
                     ++h->launches;
                     for (int t = 0; t < T; ++t) {
@@ -549,6 +562,7 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                 o_final = xf[T & 1];
             }
             if ((phase_mask & 4u) && !update_fused) {
+                NvtxRange range("mona.update");
                 MONA_CUDA(h, launch_update(ptrs, C, tc, vec4, o_final, b.e, b.slab_len, b.slabs, eta_lambda, eta_gamma, stream));
                 ++h->launches;
             }
@@ -641,14 +655,13 @@ mona_status mona_selftest_timeout(mona_handle* h, void* stream_v) {
         if (!b.tc_ok) continue;
         // one X X^T phase over the first matrix slot of the workspace whose stages expect 16 bytes too many
         uint8_t* ctrl = h->ws + WS_CTRL_OFF;
-        uint8_t* data = h->ws + WS_DATA_OFF;
         unsigned int* sched = (unsigned int*)(ctrl + CTRL_SCHED_OFF);
         NsProgram g{};
         g.C = 1; g.P = 1; g.delay = 1; g.inv_norm = (const float*)(ctrl + CTRL_INVNORM_OFF); g.work_counter = sched; g.done = sched + 64;
         g.selftest_extra_tx = 16;
         NsPhase& p = g.ph[0];
         p.M = p.N = (int)b.s; p.K = (int)b.l; p.a_map = p.b_map = MAP_X0; p.a_mn = p.b_mn = b.tall ? 1 : 0; p.symmetric = 1; p.ab_same = 1;
-        p.d = (__nv_bfloat16*)(data + b.off_a); p.ld = b.s; p.mat_stride = b.s * b.s; p.c1 = 0.f; p.c2 = 1.f;
+        p.d_map = MAP_A; p.ld = b.s; p.mat_stride = b.s * b.s; p.c1 = 0.f; p.c2 = 1.f;
         ns_phase_plan(p);
         ns_program_plan(g);
         MONA_CUDA(h, cudaMemsetAsync(sched, 0, sizeof(unsigned int) * ns_sched_words(1, 1), (cudaStream_t)stream_v));

@@ -21,10 +21,11 @@
 //   warp 1     owner of tensor memory; in the leader its lane 0 issues the MMAs and commits them to
 //              the "empty" barriers of both CTAs (multicast commit),
 //   warps 2-9  epilogue: tcgen05.ld the CTA's 128 x 256 fp32 accumulator, apply the polynomial term
-//              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, and store bf16 rows straight from
-//              registers (each thread owns 64 consecutive columns of one row, i.e. whole 128-byte lines);
+//              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, pack to bf16 into swizzled shared
+//              memory and hand the boxes to TMA stores (a thread owns one row, so storing from registers
+//              would touch 32 lines per warp instruction; the TMA writes whole lines);
 //              for the last X' = B' X of a step the same warps apply the parameter update of Eq. muon_update
-//              to the fp32 weights instead.  Then they count the item as done.
+//              to the fp32 weights instead.  When the item's stores have completed they count it as done.
 // Tensor memory holds two 256-column accumulators.  Plain tiles alternate between them, so the epilogue of one
 // tile overlaps the main loop of the next.  A macro-tile uses both at once, two neighbouring tiles computed
 // from ONE staged slice of the A operand: 96 KiB instead of 128 KiB cross from L2 per k-slice and pair.
@@ -49,12 +50,13 @@ constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
 constexpr uint32_t A_STAGE_BYTES = CTA_M * TC_BK * 2;             // 16 KiB
 constexpr uint32_t B_SUB_BYTES = CTA_N * TC_BK * 2;               // 16 KiB per 256-column tile
 constexpr int EPI_COLS = 128;                                     // output columns per epilogue phase
+constexpr uint32_t EPI_BUF_BYTES = CTA_M * EPI_COLS * 2;          // 32 KiB = 2 x 2 boxes: staging buffer of the store epilogue
 constexpr uint32_t TMEM_COLS = 512;                               // 2 accumulators x 256 fp32 columns
 constexpr int STAGES = 4;                                         // operand ring depth
 constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + 2 * B_SUB_BYTES; // 48 KiB: room for a macro-tile's k-slice
 constexpr int RING = 4;                                           // published-but-unfinished work items
 constexpr uint32_t SMEM_CTRL_BYTES = 512;
-constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + SMEM_CTRL_BYTES + 1024;
+constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
 constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
 // readers of a published item: MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
 constexpr uint32_t RING_READERS = 1 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
@@ -92,15 +94,32 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// The same with the default semantics, for hand-overs that carry no shared-memory data (tensor-memory accumulators).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// CLUSTER: acquire at cluster scope, for barriers through which the peer CTA passes ordinary shared-memory data
+// (the item ring); the pipeline barriers (TMA bytes, tcgen05 commits, accumulator hand-over) use the default scope.
+template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
+    if (CLUSTER) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+    }
     return ok != 0;
 }
 __device__ __forceinline__ void latch_timeout(volatile int* abort_flag, DeviceStatus* status, unsigned site) {
@@ -109,13 +128,14 @@ __device__ __forceinline__ void latch_timeout(volatile int* abort_flag, DeviceSt
     status->timeout_site = site;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
                                           unsigned site) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
     const long long t0 = clock64();
     unsigned spins = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
@@ -176,6 +196,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all earlier store groups of this thread have finished READING shared memory (the staging buffer may be rewritten)
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all earlier store groups of this thread have completed (their global writes are done)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Orders this thread's earlier generic-proxy accesses (plain loads/stores, acquire loads) with later accesses
 // through the asynchronous proxy (TMA), and the other way round.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -316,7 +346,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const __grid_constant__ UpdateTable upd, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzle atoms need 1024-byte alignment
-    const uint32_t ctrl = base + STAGES * STAGE_BYTES;
+    const uint32_t epi_buf = base + STAGES * STAGE_BYTES;
+    const uint32_t ctrl = epi_buf + EPI_BUF_BYTES;
     const uint32_t bar_full = ctrl;                             // STAGES x 8 B (used in the leader)
     const uint32_t bar_empty = bar_full + 8 * STAGES;           // STAGES x 8 B
     const uint32_t bar_acc_full = bar_empty + 8 * STAGES;       // 2 x 8 B, one per accumulator
@@ -357,7 +388,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const uint32_t ring_empty_leader = map_to_cta(bar_ring_empty, 0);
     auto take_item = [&](unsigned n, Item& it, unsigned site, bool arrive) -> bool {
         const uint32_t slot = n % RING, par = (n / RING) & 1u;
-        if (!mbar_wait(bar_ring_full + 8 * slot, par, abort_flag, status, site)) return false;
+        if (!mbar_wait<true>(bar_ring_full + 8 * slot, par, abort_flag, status, site)) return false;
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(it.c), "=r"(it.q), "=r"(it.t), "=r"(it.stop) : "r"(ring_items + 16 * slot) : "memory");
         if (arrive) mbar_arrive_cluster(ring_empty_leader + 8 * slot);
         return true;
@@ -439,7 +470,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     if (!ok) break;
                 }
                 const uint32_t slot = published % RING, par = (published / RING) & 1u;
-                if (!(ok = mbar_wait(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
+                if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
                 asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
                 mbar_arrive_cluster(ring_full_own + 8 * slot);
@@ -529,6 +560,11 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         const int row_in_cta = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
+        const bool issuer = threadIdx.x == 64;                 // first epilogue thread: issues and retires TMA stores
+        // position of this thread's row inside the staging buffer: box (row half, column half), 128-byte rows
+        const uint32_t box_row = (uint32_t)(row_in_cta & 63);
+        const uint32_t stage_off = (uint32_t)(((row_in_cta >> 6) * 2 + half)) * BOX_BYTES + box_row * 128u;
+        const uint32_t swz = box_row & 7u;
         uint32_t acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
         bool alive = true;
         for (unsigned n = 0; alive; ++n) {
@@ -540,6 +576,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             if (lane == 0) mbar_arrive_cluster(ring_empty_leader + 8 * (n % RING));   // every lane has its copy of the item
             if (it.stop) break;
             const NsPhase& p = g.ph[it.q];
+            const CUtensorMap* tma_d = &maps.m[p.d_map];
             const TileCoord tc = decode_tile(p, it.t);
             const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
             const int gr = m0 + row_in_cta;
@@ -549,6 +586,26 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             if (p.post_mode) { const float sc = g.inv_norm[it.c]; post = p.post_mode == 2 ? sc * sc : sc; }
             const float c1 = p.c1 * post, c2 = p.c2 * post;
             const uint32_t acc0 = tc.nsub == 2 ? 0u : acc_next;
+            // 128 packed columns of this thread's row go to the staging buffer and from there, as four boxes, to D
+            auto stage_and_store = [&](const uint4* pk, int x0) {
+                if (issuer) bulk_wait_read();          // the stores issued for the previous phase have read the buffer
+                epi_bar_sync(1);
+                #pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const uint32_t addr = epi_buf + stage_off + (((uint32_t)q ^ swz) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q].x), "r"(pk[q].y), "r"(pk[q].z), "r"(pk[q].w) : "memory");
+                }
+                fence_proxy_async();                   // generic-proxy writes above must be visible to the TMA engine
+                epi_bar_sync(2);
+                if (issuer) {
+                    #pragma unroll
+                    for (int bx = 0; bx < 4; ++bx) {
+                        const int x = x0 + (bx & 1) * TC_BOX, y = m0 + (bx >> 1) * TC_BOX;
+                        if (x < p.N && y < p.M) tma_store_3d(tma_d, epi_buf + bx * BOX_BYTES, x, y, it.c);   // clipped at the extents
+                    }
+                    bulk_commit();
+                }
+            };
             for (int u = 0; u < tc.nsub && alive; ++u) {
                 const uint32_t acc = acc0 + u;
                 const int n0 = (tc.tn + u) * TC_BN;
@@ -571,17 +628,42 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 tc_fence_after();
                 acc_par ^= 1u << acc;
                 const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
+                auto release_acc = [&]() {
+                    // this warp has read all it needs from the accumulator: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
+                };
+                if (!p.cin && !p.fuse_update && p.diag_add == 0.f) {
+                    // no axpy operand, no diagonal term (X' = B' X and X X^T): a thread's share of the accumulator fits in 64
+                    // packed registers, so read and pack all of it, release the accumulator, and only then stage and store.
+                    // For a macro-tile, whose epilogue nothing hides, this keeps the tensor cores' wait short.
+                    uint4 pk[2][8];
+                    #pragma unroll
+                    for (int ph = 0; ph < 2; ++ph) {
+                        if (ph < nphases) {
+                            float v[64];
+                            tmem_ld32(t_base + ph * EPI_COLS, v);
+                            tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
+                            tmem_ld_wait();
+                            #pragma unroll
+                            for (int j = 0; j < 64; ++j) v[j] *= c2;
+                            #pragma unroll
+                            for (int q = 0; q < 8; ++q) pk[ph][q] = pack8(v + 8 * q);
+                        }
+                    }
+                    release_acc();
+                    #pragma unroll
+                    for (int ph = 0; ph < 2; ++ph)
+                        if (ph < nphases) stage_and_store(pk[ph], n0 + ph * EPI_COLS);
+                    continue;
+                }
                 for (int ph = 0; ph < nphases; ++ph) {
                     float v[64];
                     tmem_ld32(t_base + ph * EPI_COLS, v);
                     tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
                     tmem_ld_wait();
-                    if (ph == nphases - 1) {
-                        // this warp has read all it needs from the accumulator: hand it back to the MMA issuer
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_cluster(acc_empty_leader + 8 * acc);
-                    }
+                    if (ph == nphases - 1) release_acc();
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
                     if (p.cin) {
                         const uint32_t w[32] = {cin_raw[0].x, cin_raw[0].y, cin_raw[0].z, cin_raw[0].w, cin_raw[1].x, cin_raw[1].y,
@@ -604,13 +686,12 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         #pragma unroll
                         for (int j = 0; j < 64; ++j) v[j] += (gc0 + j == gr) ? p.diag_add : 0.f;
                     }
-                    if (!row_ok) continue;
                     if (!p.fuse_update) {
-                        __nv_bfloat16* drow = p.d + row_off + gc0;
+                        uint4 pk[8];
                         #pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            if (gc0 + 8 * q < p.N) *reinterpret_cast<uint4*>(drow + 8 * q) = pack8(v + 8 * q);
-                    } else {
+                        for (int q = 0; q < 8; ++q) pk[q] = pack8(v + 8 * q);
+                        stage_and_store(pk, n0 + ph * EPI_COLS);
+                    } else if (row_ok) {
                         // Eq. muon_update on this thread's 64 parameters: W <- (W - eta lambda W) - eta gamma O
                         float* wrow = upd.w[it.c] + (long long)gr * p.ld + gc0;
                         float* orow = upd.o[it.c] ? upd.o[it.c] + (long long)gr * p.ld + gc0 : nullptr;
@@ -630,15 +711,18 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             }
             if (!alive) break;
             if (tc.nsub == 1) acc_next ^= 1u;
-            // count the item as done for its matrix and phase: every thread's stores, fenced, then one arrival per CTA
+            // count the item as done for its matrix and phase once its output is in global memory: the TMA stores have
+            // completed (issuer) and every thread's own stores are fenced; then one arrival per CTA
+            if (issuer) bulk_wait_all();
             fence_proxy_async();
             __threadfence();
             epi_bar_sync(1);
-            if (threadIdx.x == 64) {
+            if (issuer) {
                 __threadfence();
                 atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
             }
         }
+        if (issuer) bulk_wait_all();           // shared memory must outlive the stores that read it
     }
 
     if (*abort_flag) __nanosleep(200000);      // let copies that are still in flight land before the CTA goes away

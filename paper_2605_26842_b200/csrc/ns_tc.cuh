@@ -17,8 +17,8 @@ constexpr int NS_MAPS = 4;          // operand tensors of a chunk: X ping, X pon
 
 // One batched GEMM ("phase") of the iteration of Eq. newton_schulz over the C matrices of a chunk:
 //     D = post * (c1 * Cin + c2 * Aop x Bop^T) + diag_add * I,   D, Cin bf16; accumulation fp32.
-// Operand tiles are fetched through tensor maps over [C][rows][cols] bf16 tensors; D and Cin are addressed
-// directly.  An operand is "K-major" when k is its contiguous index and "MN-major" when its row index is
+// Operand tiles are fetched, and D is stored, through tensor maps over [C][rows][cols] bf16 tensors; Cin is
+// addressed directly.  An operand is "K-major" when k is its contiguous index and "MN-major" when its row index is
 // contiguous; tall weights use the MN-major form so that X^T X and X B' need no transposed copy.
 //
 // Symmetric matrices (X X^T, b A + c A^2 + a I) are only ever stored in their lower block triangle:
@@ -31,7 +31,7 @@ constexpr int NS_MAPS = 4;          // operand tensors of a chunk: X ping, X pon
 // straight from the fp32 accumulator, and writes D itself (fp32) only where an output pointer is given.
 struct NsPhase {
     int M, N, K;                // per-matrix GEMM extents
-    int a_map, b_map;           // which of the chunk's tensor maps the operands come from
+    int a_map, b_map, d_map;    // which of the chunk's tensor maps the operands come from and the output goes to
     int a_mn, b_mn;             // 1: operand is MN-major (ignored for an operand flagged *_sym)
     int a_sym, b_sym;           // 1: operand is a symmetric matrix stored as its lower block triangle
     int symmetric;              // 1: D = D^T, compute lower-triangle tiles only
@@ -40,9 +40,9 @@ struct NsPhase {
     int wide;                   // 1 (non-symmetric D only): a work item is a 256 x 512 macro-tile, two tiles that share
                                 //    one staged slice of the A operand, one per tensor-memory accumulator
     int tiles_m, tiles_n, items_per_mat;   // filled by ns_phase_plan(); items are macro-tiles when `wide`
-    __nv_bfloat16* d;           // output [C][M][N] (dense), unused when fuse_update
-    const __nv_bfloat16* cin;   // may be null; same layout as d; lower-block-stored when D is symmetric
-    long long ld, mat_stride;   // leading dimension and per-matrix stride of d and cin, in elements
+    const __nv_bfloat16* cin;   // may be null; [C][M][N] like D; lower-block-stored when D is symmetric
+    long long ld, mat_stride;   // leading dimension and per-matrix stride of cin (and of the fp32 parameter when
+                                // fuse_update), in elements
     float c1, c2;
     float diag_add;             // added to D(i,i): folds the a*X term of the quintic into B' = b A + c A^2 + a I
     int post_mode;              // 0: post = 1, 1: post = inv_norm[c], 2: post = inv_norm[c]^2
