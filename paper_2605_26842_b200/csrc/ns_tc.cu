@@ -14,9 +14,10 @@
 // stream, issued by the even CTA (the "leader"), drives the tensor cores of both SMs.  Each CTA stages its own
 // 128 rows of the A operand and its own 128 rows of the B operand per k-slice, so a pair moves 64 KiB from L2
 // per 256 x 256 x 64 step (half of what two independent 128 x 256 tiles would).  Roles inside a CTA:
-//   warp 0     lane 0 of the leader: scheduler (takes items, waits for their dependencies, publishes them to
-//              both CTAs through a small ring in shared memory) and TMA producer; lane 0 of the peer: TMA
-//              producer.  Operand boxes go into a ring of shared-memory stages; the copies of both CTAs
+//   warp 10    (leader only) scheduler: takes items from the counter, waits for their dependencies and publishes them
+//              to both CTAs through a small ring in shared memory, a few items ahead of the pipeline, so that the
+//              round trips to the counters never hold up a copy,
+//   warp 0     TMA producer: operand boxes into a ring of shared-memory stages; the copies of both CTAs
 //              complete on the leader's "full" barrier,
 //   warp 1     owner of tensor memory; in the leader its lane 0 issues the MMAs and commits them to
 //              the "empty" barriers of both CTAs (multicast commit),
@@ -41,8 +42,9 @@ namespace {
 
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
-constexpr int TC_THREADS = 64 + TC_EPI_THREADS;
-// registers are granted to warps in groups of four: 10 warps count as 12, and 12 x 32 x 168 fits the SM's 64 K
+constexpr int SCHED_WARP = 2 + TC_EPI_WARPS;                      // warp 10: the scheduler (leader CTA)
+constexpr int TC_THREADS = 64 + TC_EPI_THREADS + 32;
+// registers are granted to warps in groups of four: 11 warps count as 12, and 12 x 32 x 168 fits the SM's 64 K
 constexpr int TC_MAX_REGS = 168;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
@@ -58,10 +60,10 @@ constexpr int RING = 4;                                           // published-b
 constexpr uint32_t SMEM_CTRL_BYTES = 512;
 constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
 constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
-// readers of a published item: MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
-constexpr uint32_t RING_READERS = 1 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
+// readers of a published item: producer + MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
+constexpr uint32_t RING_READERS = 2 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
 static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-static_assert(8 * (2 * STAGES + 4 + 2 * RING) + 16 + 16 * RING <= SMEM_CTRL_BYTES, "control block");
+static_assert(8 * (2 * STAGES + 4 + 2 * RING) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -210,6 +212,22 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // through the asynchronous proxy (TMA), and the other way round.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
+// Shared-memory matrix descriptor (64 bits) for a 128-byte-swizzled bf16 tile whose rows are 128 bytes long and
+// stacked densely (what a 64-wide TMA box with SWIZZLE_128B produces):
+//   bits [0,14)  start address >> 4            bits [16,30) leading byte offset >> 4
+//   bits [32,46) stride byte offset >> 4       bit 46       descriptor version for sm_100      bits [61,64) layout: 2 = 128-byte swizzle
+//   K-major : row = m/n index, 128 B = 64 k.  Groups of 8 rows are 1024 B apart (stride byte offset);
+//             the leading byte offset is not used by swizzled K-major layouts (encoded 1).
+//   MN-major: row = k index, 128 B = 64 m/n.  Groups of 8 k-rows are 1024 B apart (stride byte offset);
+//             the next 64 m/n lives in the next 8 KiB box (leading byte offset).
+// Shared-memory addresses are below 256 KiB, so address >> 4 fits its field and the low word is address >> 4 | offset field.
+constexpr uint32_t DESC_LBO_K = 1u << 16;
+constexpr uint32_t DESC_LBO_MN = (BOX_BYTES >> 4) << 16;
+constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+// Instruction descriptor, kind::f16: D fp32 (bit 4), A and B bf16 (bits 7, 10), N >> 3 at bit 17, M >> 4 at bit 24 (M = 256 over
+// the pair, N = 256); bits 15 / 16 say that A / B is MN-major.
+constexpr uint32_t IDESC_BASE = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TC_BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+
 // ---- tcgen05 --------------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
@@ -230,13 +248,16 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
                  : "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem]^T over the CTA pair, bf16 inputs, fp32 accumulate; accumulate == 0 overwrites D.
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+// The two shared-memory matrix descriptors are given by their low words; the high word is the same for every operand.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint32_t a_desc_lo, uint32_t b_desc_lo, uint32_t idesc,
                                             uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "mov.b64 da, {%1, %5};\n\t"
+        "mov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_desc_lo), "r"(b_desc_lo), "r"(idesc), "r"(accumulate), "r"(DESC_HI)
         : "memory");
 }
 // 32 lanes x 32 consecutive fp32 columns: thread t of the warp receives row (lane base + t).
@@ -254,30 +275,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor for a 128-byte-swizzled bf16 tile whose rows are 128 bytes long and
-// stacked densely (what a 64-wide TMA box with SWIZZLE_128B produces).
-//   K-major : row = m/n index, 128 B = 64 k.  Groups of 8 rows are 1024 B apart (stride byte offset);
-//             the leading byte offset is not used by swizzled K-major layouts (encoded 1).
-//   MN-major: row = k index, 128 B = 64 m/n.  Groups of 8 k-rows are 1024 B apart (stride byte offset);
-//             the next 64 m/n lives in the next 8 KiB box (leading byte offset).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fffu);                                  // start address, bits [0,14)
-    d |= (uint64_t)(mn_major ? (BOX_BYTES >> 4) : 1u) << 16;                 // leading byte offset, bits [16,30)
-    d |= (uint64_t)(1024u >> 4) << 32;                                       // stride byte offset, bits [32,46)
-    d |= (uint64_t)1 << 46;                                                  // descriptor version for sm_100
-    d |= (uint64_t)2 << 61;                                                  // layout: 128-byte swizzle
-    return d;
-}
-// Instruction descriptor, kind::f16: D fp32, A and B bf16, M = 256 over the pair, N = 256.
-__device__ __forceinline__ uint32_t instr_desc(int a_mn, int b_mn) {
-    return (1u << 4)                      // D format fp32
-           | (1u << 7) | (1u << 10)       // A, B format bf16
-           | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
-           | ((uint32_t)(TC_BN >> 3) << 17)
-           | ((uint32_t)(TC_BM >> 4) << 24);
-}
 
 // A published work item: item `t` of phase `q` for matrix `c`; stop != 0 ends the role loops.
 struct Item {
@@ -356,6 +353,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const uint32_t bar_ring_empty = bar_ring_full + 8 * RING;   // RING x 8 B (used in the leader)
     const uint32_t tmem_slot = bar_ring_empty + 8 * RING;       // 4 B + abort flag 4 B + 8 B pad
     const uint32_t ring_items = tmem_slot + 16;                 // RING x 16 B
+    volatile unsigned int* phase_items = reinterpret_cast<volatile unsigned int*>(smem_raw + (ring_items + 16 * RING - smem_u32(smem_raw)));   // NS_MAX_PHASES x 4 B
     uint8_t* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + (tmem_slot - ctrl));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + (tmem_slot - ctrl) + 4);
@@ -366,6 +364,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        for (int q = 0; q < NS_MAX_PHASES; ++q) phase_items[q] = q < P ? (unsigned)g.ph[q].items_per_mat : 0u;
         for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
@@ -438,55 +437,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     };
 
     if (warp == 0) {
-        if (lane == 0 && rank == 0) {
-            // ---------------- scheduler + TMA producer (leader) ----------------
-            const uint32_t ring_items_peer = map_to_cta(ring_items, 1), ring_full_peer = map_to_cta(bar_ring_full, 1);
-            const uint32_t ring_full_own = map_to_cta(bar_ring_full, 0);
-            int cur_tau = 0, cur_q = 0;                // group (tau, q) of the item order the cursor stands in
-            unsigned cur_base = 0;                     // index of the first item of that group
-            unsigned published = 0;
-            unsigned idx = atomicAdd(g.work_counter, 1u);
-            bool ok = true;
-            while (ok) {
-                Item it;
-                it.c = it.q = it.t = 0;
-                it.stop = idx >= g.total_items ? 1 : 0;
-                unsigned next_idx = 0;
-                if (!it.stop) {
-                    next_idx = atomicAdd(g.work_counter, 1u);      // in flight while this item is being staged
-                    // item order: for tau = 0, 1, ...: for q = 0 .. P-1: matrix c = tau - delay * q (if it exists): its items
-                    while (true) {
-                        const int c = cur_tau - g.delay * cur_q;
-                        const unsigned n = (c >= 0 && c < g.C) ? (unsigned)g.ph[cur_q].items_per_mat : 0u;
-                        if (idx < cur_base + n) { it.c = c; it.q = cur_q; it.t = (int)(idx - cur_base); break; }
-                        cur_base += n;
-                        if (++cur_q == P) { cur_q = 0; ++cur_tau; }
-                    }
-                    // the phase before it must be complete for this matrix: its outputs are this item's operands, and the
-                    // buffers this item overwrites were last read two phases further back
-                    if (it.q > 0)
-                        ok = wait_counter(g.done + (size_t)it.c * P + (it.q - 1), 2u * (unsigned)g.ph[it.q - 1].items_per_mat, abort_flag, status, 6);
-                    fence_proxy_async();
-                    if (!ok) break;
-                }
-                const uint32_t slot = published % RING, par = (published / RING) & 1u;
-                if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
-                asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
-                mbar_arrive_cluster(ring_full_own + 8 * slot);
-                mbar_arrive_cluster(ring_full_peer + 8 * slot);
-                ++published;
-                if (it.stop) break;
-                ok = produce(it);
-                idx = next_idx;
-            }
-            // stay until the tensor cores have released every stage: the commits arrive on this CTA's barriers
-            for (int s = 0; s < STAGES && ok; ++s) {
-                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-            }
-        } else if (lane == 0) {
-            // ---------------- TMA producer (peer) ----------------
+        if (lane == 0) {
+            // ---------------- TMA producer (both CTAs) ----------------
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
@@ -494,6 +446,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 fence_proxy_async();       // the scheduler's acquire of the dependency precedes these copies
                 ok = produce(it);
             }
+            // stay until the tensor cores have released every stage: the commits arrive on this CTA's barriers
             for (int s = 0; s < STAGES && ok; ++s) {
                 ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -512,34 +465,51 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const bool shared_ab = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
                 const uint32_t acc0 = tc.nsub == 2 ? 0u : acc_next;
                 const int num_kb = (p.K + TC_BK - 1) / TC_BK;
-                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                // This one thread feeds both tensor cores, so the loop over k-slices is kept to a few dozen instructions:
+                // everything that does not change inside a tile is worked out here.  An operand is MN-major from the k-slice
+                // `switch` on (0: always, num_kb: never; a symmetric operand turns MN-major where it crosses its diagonal block).
+                const int a_switch = p.a_sym ? (tc.tm + 1) * (TC_BM / TC_BK) : (p.a_mn ? 0 : num_kb);
+                int b_switch[2];
+                #pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    b_switch[u] = shared_ab ? a_switch : (p.b_sym ? (tc.tn + u + 1) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb));
+                const uint32_t b_off0 = shared_ab ? 0u : (A_STAGE_BYTES >> 4);             // operand offsets inside a stage, in 16-byte units
+                const uint32_t b_off1 = (A_STAGE_BYTES + B_SUB_BYTES) >> 4;
+                // the accumulators must have been drained by the epilogue of their previous tile
+                for (int u = 0; u < tc.nsub && ok; ++u)
+                    ok = mbar_wait(bar_acc_empty + 8 * (acc0 + u), ((acc_par >> (acc0 + u)) & 1u) ^ 1u, abort_flag, status, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base + acc0 * TC_BN, d1 = d0 + TC_BN;
+                uint32_t accum = 0u;
+                uint32_t stage_lo = (base + mstage * STAGE_BYTES) >> 4;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    // no tcgen05 fence here: the operands arrive through the asynchronous proxy and the barrier orders them
                     if (!(ok = mbar_wait(bar_full + 8 * mstage, mphase, abort_flag, status, 3))) break;
-                    tc_fence_after();
-                    const int k0 = kb * TC_BK;
-                    const int a_mn = p.a_sym ? fetch_transposed(1, tc.tm, k0) : p.a_mn;
+                    const uint32_t a_mn = kb >= a_switch ? 1u : 0u, b_mn0 = kb >= b_switch[0] ? 1u : 0u;
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
-                    const uint32_t a_kstep = a_mn ? (2048u >> 4) : (32u >> 4);
-                    const uint32_t sa = base + mstage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
-                    const uint64_t da = smem_desc(sa, a_mn);
-                    for (int u = 0; u < tc.nsub; ++u) {
-                        const uint32_t acc = acc0 + u;
-                        if (kb == 0) {     // the epilogue must have drained this accumulator's previous tile
-                            if (!(ok = mbar_wait(bar_acc_empty + 8 * acc, ((acc_par >> acc) & 1u) ^ 1u, abort_flag, status, 2))) break;
-                            tc_fence_after();
-                        }
-                        const int b_mn = shared_ab ? a_mn : (p.b_sym ? fetch_transposed(1, tc.tn + u, k0) : p.b_mn);
-                        const uint32_t b_kstep = b_mn ? (2048u >> 4) : (32u >> 4);
-                        const uint64_t db = smem_desc(shared_ab ? sa : sb + u * B_SUB_BYTES, b_mn);
-                        const uint32_t idesc = instr_desc(a_mn, b_mn);
-                        const uint32_t d_tmem = tmem_base + acc * TC_BN;
-                        #pragma unroll
-                        for (int k = 0; k < TC_BK / 16; ++k)
-                            tc_mma_bf16(d_tmem, da + (uint64_t)(k * a_kstep), db + (uint64_t)(k * b_kstep), idesc,
-                                        (kb | k) != 0 ? 1u : 0u);
+                    const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step0 = b_mn0 ? (2048u >> 4) : (32u >> 4);
+                    const uint32_t a_lo = stage_lo | (a_mn ? DESC_LBO_MN : DESC_LBO_K);
+                    const uint32_t b_lo0 = (stage_lo + b_off0) | (b_mn0 ? DESC_LBO_MN : DESC_LBO_K);
+                    const uint32_t idesc0 = IDESC_BASE | (a_mn << 15) | (b_mn0 << 16);
+                    #pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k) {
+                        tc_mma_bf16(d0, a_lo + k * a_step, b_lo0 + k * b_step0, idesc0, accum);
+                        accum = 1u;
                     }
-                    if (!ok) break;
+                    if (tc.nsub == 2) {
+                        const uint32_t b_mn1 = kb >= b_switch[1] ? 1u : 0u;
+                        const uint32_t b_step1 = b_mn1 ? (2048u >> 4) : (32u >> 4);
+                        const uint32_t b_lo1 = (stage_lo + b_off1) | (b_mn1 ? DESC_LBO_MN : DESC_LBO_K);
+                        const uint32_t idesc1 = IDESC_BASE | (a_mn << 15) | (b_mn1 << 16);
+                        const uint32_t accum1 = kb != 0 ? 1u : 0u;
+                        tc_mma_bf16(d1, a_lo, b_lo1, idesc1, accum1);
+                        #pragma unroll
+                        for (int k = 1; k < TC_BK / 16; ++k) tc_mma_bf16(d1, a_lo + k * a_step, b_lo1 + k * b_step1, idesc1, 1u);
+                    }
                     tc_commit_pair(bar_empty + 8 * mstage);     // frees the stage in both CTAs when these MMAs have read it
-                    if (++mstage == STAGES) { mstage = 0; mphase ^= 1u; }
+                    stage_lo += STAGE_BYTES >> 4;
+                    if (++mstage == STAGES) { mstage = 0; mphase ^= 1u; stage_lo = base >> 4; }
                 }
                 if (!ok) break;
                 for (int u = 0; u < tc.nsub; ++u) {
@@ -548,6 +518,60 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     acc_par ^= 1u << acc;
                 }
                 if (tc.nsub == 1) acc_next ^= 1u;
+            }
+        }
+    } else if (warp == SCHED_WARP) {
+        if (lane == 0 && rank == 0) {
+            // ---------------- scheduler (leader CTA only) ----------------
+            const uint32_t ring_items_peer = map_to_cta(ring_items, 1), ring_full_peer = map_to_cta(bar_ring_full, 1);
+            const uint32_t ring_full_own = map_to_cta(bar_ring_full, 0);
+            // Item order: for tau = 0, 1, ...: for q = 0 .. P-1: the items of phase q of matrix c = tau - delay * q, where that
+            // matrix exists.  The cursor (tau, q, index of the group's first item) only moves forward; per-phase item counts
+            // come from shared memory, and the q range that has a matrix at this tau is computed, not searched.
+            int cur_tau = 0, cur_q = 0;
+            unsigned cur_base = 0;
+            auto decode = [&](unsigned idx, Item& it) {
+                it.stop = idx >= g.total_items ? 1 : 0;
+                it.c = it.q = it.t = 0;
+                if (it.stop) return;
+                while (true) {
+                    const int over = cur_tau - g.C + 1;                                 // c < C  <=>  q >= over / delay (rounded up)
+                    const int q_lo = over > 0 ? (over + g.delay - 1) / g.delay : 0;
+                    int q_hi = cur_tau / g.delay;                                        // c >= 0
+                    if (q_hi > P - 1) q_hi = P - 1;
+                    if (cur_q < q_lo) cur_q = q_lo;
+                    if (cur_q > q_hi) { ++cur_tau; cur_q = 0; continue; }
+                    const unsigned n = phase_items[cur_q];
+                    if (idx < cur_base + n) { it.c = cur_tau - g.delay * cur_q; it.q = cur_q; it.t = (int)(idx - cur_base); return; }
+                    cur_base += n;
+                    ++cur_q;
+                }
+            };
+            // The phase before an item must be complete for its matrix: its outputs are the item's operands, and the buffers
+            // the item overwrites were last read two phases further back.
+            auto dependency = [&](const Item& it, const unsigned int*& ctr, unsigned& need) {
+                ctr = nullptr; need = 0u;
+                if (!it.stop && it.q > 0) { ctr = g.done + (size_t)it.c * P + (it.q - 1); need = 2u * phase_items[it.q - 1]; }
+            };
+            unsigned published = 0;
+            bool ok = true;
+            while (ok) {
+                // an item is taken only once a ring slot is free for it: items stay in the common pool as long as possible
+                const uint32_t slot = published % RING, par = (published / RING) & 1u;
+                if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
+                const unsigned idx = atomicAdd(g.work_counter, 1u);
+                Item it;
+                decode(idx, it);
+                const unsigned int* ctr; unsigned need;
+                dependency(it, ctr, need);
+                if (ctr && !(ok = wait_counter(ctr, need, abort_flag, status, 6))) break;
+                fence_proxy_async();
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
+                asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
+                mbar_arrive_cluster(ring_full_own + 8 * slot);
+                mbar_arrive_cluster(ring_full_peer + 8 * slot);
+                ++published;
+                if (it.stop) break;
             }
         }
     } else {
