@@ -169,11 +169,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// bf16 tensor [C][outer][inner] (inner contiguous) cut into 64 x 64 boxes with the 128-byte swizzle.
-bool encode_map(EncodeTiledFn fn, CUtensorMap* map, void* base, int64_t inner, int64_t outer, int64_t C) {
+// bf16 tensor [C][outer][inner] (inner contiguous) cut into boxes of 64 x box_rows with the 128-byte swizzle.
+bool encode_map(EncodeTiledFn fn, CUtensorMap* map, void* base, int64_t inner, int64_t outer, int64_t C, int box_rows) {
     cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)C};
     cuuint64_t strides[2] = {(cuuint64_t)inner * 2, (cuuint64_t)inner * (cuuint64_t)outer * 2};
-    cuuint32_t box[3] = {(cuuint32_t)TC_BOX, (cuuint32_t)TC_BOX, 1};
+    cuuint32_t box[3] = {(cuuint32_t)TC_BOX, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -334,9 +334,12 @@ mona_status mona_create_opt(mona_handle** out, const mona_matrix_desc* descs, in
         bool ok = true;
         for (int sl = 0; sl < NSLOTS; ++sl) {
             uint8_t* data = h->ws + WS_DATA_OFF + sl * h->plan.slot_bytes;
-            for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.maps[sl].m[MAP_X0 + i], data + b.off_x[i], b.cols, b.rows, b.Cb);
-            ok = ok && encode_map(encode, &b.maps[sl].m[MAP_A], data + b.off_a, b.s, b.s, b.Cb);
-            ok = ok && encode_map(encode, &b.maps[sl].m[MAP_B], data + b.off_b, b.s, b.s, b.Cb);
+            for (int big = 0; big < 2; ++big) {     // 64-row boxes, then 128-row boxes
+                const int rows = big ? 2 * TC_BOX : TC_BOX, at = big * NS_TENSORS;
+                for (int i = 0; i < 2; ++i) ok = ok && encode_map(encode, &b.maps[sl].m[at + MAP_X0 + i], data + b.off_x[i], b.cols, b.rows, b.Cb, rows);
+                ok = ok && encode_map(encode, &b.maps[sl].m[at + MAP_A], data + b.off_a, b.s, b.s, b.Cb, rows);
+                ok = ok && encode_map(encode, &b.maps[sl].m[at + MAP_B], data + b.off_b, b.s, b.s, b.Cb, rows);
+            }
         }
         if (!ok) return h->fail(MONA_ERR_CUDA, "cuTensorMapEncodeTiled failed for bucket %lldx%lld", (long long)b.rows, (long long)b.cols);
     }

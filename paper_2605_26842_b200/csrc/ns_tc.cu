@@ -399,35 +399,48 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     auto produce = [&](const Item& it) -> bool {
         const NsPhase& p = g.ph[it.q];
         const TileCoord tc = decode_tile(p, it.t);
-        const CUtensorMap* tma_a = &maps.m[p.a_map];
-        const CUtensorMap* tma_b = &maps.m[p.b_map];
+        // K-major operands come as one box of 128 rows, MN-major ones as two boxes of 64 (the swizzle row is 64 elements)
+        const CUtensorMap* a_box64 = &maps.m[p.a_map];
+        const CUtensorMap* a_box128 = &maps.m[p.a_map + NS_TENSORS];
+        const CUtensorMap* b_box64 = &maps.m[p.b_map];
+        const CUtensorMap* b_box128 = &maps.m[p.b_map + NS_TENSORS];
         const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;      // this CTA's rows of the A operand
         const int n0 = tc.tn * TC_BN + (int)rank * CTA_N;      // this CTA's rows of the B operand (first sub-tile)
         // diagonal tile of X X^T or A A: both operands are the same rows, staged once
         const bool shared_ab = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
-        const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (shared_ab ? 0u : (uint32_t)tc.nsub * B_SUB_BYTES)) + (uint32_t)g.selftest_extra_tx;
+        const int nb = shared_ab ? 0 : tc.nsub;
+        const uint32_t tx_bytes = 2u * (A_STAGE_BYTES + (uint32_t)nb * B_SUB_BYTES) + (uint32_t)g.selftest_extra_tx;
         const int num_kb = (p.K + TC_BK - 1) / TC_BK;
+        // from k-slice `switch` on the operand is MN-major (see the MMA issuer)
+        const int a_switch = p.a_sym ? (tc.tm + 1) * (TC_BM / TC_BK) : (p.a_mn ? 0 : num_kb);
+        const int b_switch0 = p.b_sym ? (tc.tn + 1) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb);
+        const int b_switch1 = p.b_sym ? (tc.tn + 2) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb);
         for (int kb = 0; kb < num_kb; ++kb) {
             if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1)) return false;
             const uint32_t full = full_leader + 8 * stage;
-            const uint32_t sa = base + stage * STAGE_BYTES, sb = sa + A_STAGE_BYTES;
+            const uint32_t sa = base + stage * STAGE_BYTES;
             const int k0 = kb * TC_BK;
             if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx_bytes);   // both CTAs' copies land here
-            const int a_mn = p.a_sym ? fetch_transposed(1, tc.tm, k0) : p.a_mn;
-            #pragma unroll
-            for (int j = 0; j < CTA_M / TC_BOX; ++j) {
-                if (a_mn) tma_load_3d(sa + j * BOX_BYTES, tma_a, full, m0 + j * TC_BOX, k0, it.c);
-                else      tma_load_3d(sa + j * BOX_BYTES, tma_a, full, k0, m0 + j * TC_BOX, it.c);
+            if (kb >= a_switch) {
+                tma_load_3d(sa, a_box64, full, m0, k0, it.c);
+                tma_load_3d(sa + BOX_BYTES, a_box64, full, m0 + TC_BOX, k0, it.c);
+            } else {
+                tma_load_3d(sa, a_box128, full, k0, m0, it.c);
             }
-            if (!shared_ab) {
-                for (int u = 0; u < tc.nsub; ++u) {
-                    const int b_mn = p.b_sym ? fetch_transposed(1, tc.tn + u, k0) : p.b_mn;
-                    const int nu = n0 + u * TC_BN;
-                    const uint32_t sbu = sb + u * B_SUB_BYTES;
-                    #pragma unroll
-                    for (int j = 0; j < CTA_N / TC_BOX; ++j) {
-                        if (b_mn) tma_load_3d(sbu + j * BOX_BYTES, tma_b, full, nu + j * TC_BOX, k0, it.c);
-                        else      tma_load_3d(sbu + j * BOX_BYTES, tma_b, full, k0, nu + j * TC_BOX, it.c);
+            if (nb > 0) {
+                const uint32_t sb = sa + A_STAGE_BYTES;
+                if (kb >= b_switch0) {
+                    tma_load_3d(sb, b_box64, full, n0, k0, it.c);
+                    tma_load_3d(sb + BOX_BYTES, b_box64, full, n0 + TC_BOX, k0, it.c);
+                } else {
+                    tma_load_3d(sb, b_box128, full, k0, n0, it.c);
+                }
+                if (nb > 1) {
+                    if (kb >= b_switch1) {
+                        tma_load_3d(sb + B_SUB_BYTES, b_box64, full, n0 + TC_BN, k0, it.c);
+                        tma_load_3d(sb + B_SUB_BYTES + BOX_BYTES, b_box64, full, n0 + TC_BN + TC_BOX, k0, it.c);
+                    } else {
+                        tma_load_3d(sb + B_SUB_BYTES, b_box128, full, k0, n0 + TC_BN, it.c);
                     }
                 }
             }
@@ -585,10 +598,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
         const bool issuer = threadIdx.x == 64;                 // first epilogue thread: issues and retires TMA stores
-        // position of this thread's row inside the staging buffer: box (row half, column half), 128-byte rows
-        const uint32_t box_row = (uint32_t)(row_in_cta & 63);
-        const uint32_t stage_off = (uint32_t)(((row_in_cta >> 6) * 2 + half)) * BOX_BYTES + box_row * 128u;
-        const uint32_t swz = box_row & 7u;
+        // position of this thread's row inside the staging buffer: one 128-row box per column half, 128-byte rows
+        const uint32_t stage_off = (uint32_t)half * (2u * BOX_BYTES) + (uint32_t)row_in_cta * 128u;
+        const uint32_t swz = (uint32_t)row_in_cta & 7u;
         uint32_t acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
         bool alive = true;
         for (unsigned n = 0; alive; ++n) {
@@ -600,7 +612,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             if (lane == 0) mbar_arrive_cluster(ring_empty_leader + 8 * (n % RING));   // every lane has its copy of the item
             if (it.stop) break;
             const NsPhase& p = g.ph[it.q];
-            const CUtensorMap* tma_d = &maps.m[p.d_map];
+            const CUtensorMap* tma_d = &maps.m[p.d_map + NS_TENSORS];     // 64 columns x 128 rows per store
             const TileCoord tc = decode_tile(p, it.t);
             const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
             const int gr = m0 + row_in_cta;
@@ -623,9 +635,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 epi_bar_sync(2);
                 if (issuer) {
                     #pragma unroll
-                    for (int bx = 0; bx < 4; ++bx) {
-                        const int x = x0 + (bx & 1) * TC_BOX, y = m0 + (bx >> 1) * TC_BOX;
-                        if (x < p.N && y < p.M) tma_store_3d(tma_d, epi_buf + bx * BOX_BYTES, x, y, it.c);   // clipped at the extents
+                    for (int bx = 0; bx < 2; ++bx) {
+                        const int x = x0 + bx * TC_BOX;
+                        if (x < p.N && m0 < p.M) tma_store_3d(tma_d, epi_buf + bx * 2 * BOX_BYTES, x, m0, it.c);   // clipped at the extents
                     }
                     bulk_commit();
                 }

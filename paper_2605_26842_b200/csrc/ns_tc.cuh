@@ -11,9 +11,10 @@ namespace mona {
 constexpr int TC_BM = 256;      // rows of D per tile: one CTA pair, 128 rows per CTA (UMMA M = 256)
 constexpr int TC_BN = 256;      // columns of D per tile (UMMA N = 256, each CTA stages 128 of them)
 constexpr int TC_BK = 64;       // k-slice per pipeline stage: 64 bf16 = one 128-byte swizzle row
-constexpr int TC_BOX = 64;      // every TMA box is 64 (contiguous) x 64 (strided) bf16 = 8 KiB
+constexpr int TC_BOX = 64;      // every TMA box is 64 bf16 wide (one 128-byte swizzle row) and 64 or 128 rows high
 constexpr int NS_MAX_PHASES = 15;   // 3 GEMMs x 5 iterations per launch; longer iterations take several launches
-constexpr int NS_MAPS = 4;          // operand tensors of a chunk: X ping, X pong, A, B'
+constexpr int NS_TENSORS = 4;       // operand tensors of a chunk: X ping, X pong, A, B'
+constexpr int NS_MAPS = 2 * NS_TENSORS;   // each with 64-row boxes (index t) and with 128-row boxes (index t + NS_TENSORS)
 
 // One batched GEMM ("phase") of the iteration of Eq. newton_schulz over the C matrices of a chunk:
 //     D = post * (c1 * Cin + c2 * Aop x Bop^T) + diag_add * I,   D, Cin bf16; accumulation fp32.
@@ -31,7 +32,7 @@ constexpr int NS_MAPS = 4;          // operand tensors of a chunk: X ping, X pon
 // straight from the fp32 accumulator, and writes D itself (fp32) only where an output pointer is given.
 struct NsPhase {
     int M, N, K;                // per-matrix GEMM extents
-    int a_map, b_map, d_map;    // which of the chunk's tensor maps the operands come from and the output goes to
+    int a_map, b_map, d_map;    // which of the chunk's tensors (0 .. NS_TENSORS-1) the operands come from and the output goes to
     int a_mn, b_mn;             // 1: operand is MN-major (ignored for an operand flagged *_sym)
     int a_sym, b_sym;           // 1: operand is a symmetric matrix stored as its lower block triangle
     int symmetric;              // 1: D = D^T, compute lower-triangle tiles only
