@@ -14,14 +14,14 @@
 // stream, issued by the even CTA (the "leader"), drives the tensor cores of both SMs.  Each CTA stages its own
 // 128 rows of the A operand and its own 128 rows of the B operand per k-slice, so a pair moves 64 KiB from L2
 // per 256 x 256 x 64 step (half of what two independent 128 x 256 tiles would).  Roles inside a CTA:
-//   warp 10    (leader only) scheduler: takes items from the counter, waits for their dependencies and publishes them
+//   warp 2     (leader only) scheduler: takes items from the counter, waits for their dependencies and publishes them
 //              to both CTAs through a small ring in shared memory, a few items ahead of the pipeline, so that the
 //              round trips to the counters never hold up a copy,
 //   warp 0     TMA producer: operand boxes into a ring of shared-memory stages; the copies of both CTAs
 //              complete on the leader's "full" barrier,
 //   warp 1     owner of tensor memory; in the leader its lane 0 issues the MMAs and commits them to
 //              the "empty" barriers of both CTAs (multicast commit),
-//   warps 2-9  epilogue: tcgen05.ld the CTA's 128 x 256 fp32 accumulator, apply the polynomial term
+//   warps 4-11 epilogue: tcgen05.ld the CTA's 128 x 256 fp32 accumulator, apply the polynomial term
 //              (b A + c A^2 + a I) and the deferred 1/||M||_F scale, pack to bf16 into swizzled shared
 //              memory and hand the boxes to TMA stores (a thread owns one row, so storing from registers
 //              would touch 32 lines per warp instruction; the TMA writes whole lines);
@@ -42,10 +42,15 @@ namespace {
 
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
-constexpr int SCHED_WARP = 2 + TC_EPI_WARPS;                      // warp 10: the scheduler (leader CTA)
-constexpr int TC_THREADS = 64 + TC_EPI_THREADS + 32;
-// registers are granted to warps in groups of four: 11 warps count as 12, and 12 x 32 x 168 fits the SM's 64 K
+constexpr int SCHED_WARP = 2;                                     // the scheduler (leader CTA); warp 3 has no role
+constexpr int EPI_WARP0 = 4;                                      // epilogue = warps 4..11, i.e. warpgroups 1 and 2
+constexpr int TC_THREADS = 32 * EPI_WARP0 + TC_EPI_THREADS;       // 384
+// The kernel starts with 168 registers per thread (12 warps x 32 x 168 fit the SM's 64 K); then the warpgroup of the
+// producer, MMA issuer and scheduler gives registers back and the two epilogue warpgroups take them (setmaxnreg):
+// 128 x 48 + 256 x 224 = 63488.  An epilogue thread can then hold its share of BOTH accumulators of a macro-tile.
 constexpr int TC_MAX_REGS = 168;
+constexpr int REGS_CONTROL = 48;
+constexpr int REGS_EPILOGUE = 224;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
 constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
@@ -338,7 +343,7 @@ struct UpdateTable {
     float* o[MAXC];
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(TC_MAX_REGS)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsProgram g,
                 const __grid_constant__ UpdateTable upd, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
@@ -449,6 +454,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         return true;
     };
 
+    if (warp < EPI_WARP0) {
+    // the control warpgroup gives registers back (all four warps execute this together) ...
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CONTROL));
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer (both CTAs) ----------------
@@ -587,17 +595,20 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 if (it.stop) break;
             }
         }
+    }
     } else {
-        // ---------------- epilogue (warps 2..9, both CTAs) ----------------
+        // ... and the two epilogue warpgroups take them
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_EPILOGUE));
+        // ---------------- epilogue (warps 4..11, both CTAs) ----------------
         // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4).  A 256-column
         // tile is handled in phases of 128 columns; in a phase the two warps of a quadrant take 64 columns
         // each, so a thread owns 64 consecutive columns of one row: one 128-byte line of the bf16 output.
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - EPI_WARP0) >> 2;
         const int row_in_cta = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
-        const bool issuer = threadIdx.x == 64;                 // first epilogue thread: issues and retires TMA stores
+        const bool issuer = threadIdx.x == 32 * EPI_WARP0;     // first epilogue thread: issues and retires TMA stores
         // position of this thread's row inside the staging buffer: one 128-row box per column half, 128-byte rows
         const uint32_t stage_off = (uint32_t)half * (2u * BOX_BYTES) + (uint32_t)row_in_cta * 128u;
         const uint32_t swz = (uint32_t)row_in_cta & 7u;
@@ -642,6 +653,48 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     bulk_commit();
                 }
             };
+            if (!p.cin && !p.fuse_update && p.diag_add == 0.f) {
+                // No axpy operand, no diagonal term (X X^T and X' = B' X).  A thread's share of an accumulator is 128 values,
+                // 64 registers once packed: read and pack every accumulator of the item first, handing each back to the MMA
+                // issuer as soon as it has been read, and only then stage and store.  Nothing hides the epilogue of a
+                // macro-tile, so the time the tensor cores wait is the time of these reads.
+                uint4 pk[2][2][8];
+                #pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if (u < tc.nsub) {
+                        const uint32_t acc = acc0 + u;
+                        const int n0 = (tc.tn + u) * TC_BN;
+                        bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
+                        ok = epi_bar_all(3, ok);
+                        if (!ok) { alive = false; break; }
+                        tc_fence_after();
+                        acc_par ^= 1u << acc;
+                        const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
+                        #pragma unroll
+                        for (int ph = 0; ph < 2; ++ph) {
+                            if (n0 + ph * EPI_COLS < p.N) {
+                                float v[64];
+                                tmem_ld32(t_base + ph * EPI_COLS, v);
+                                tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
+                                tmem_ld_wait();
+                                #pragma unroll
+                                for (int j = 0; j < 64; ++j) v[j] *= c2;
+                                #pragma unroll
+                                for (int q = 0; q < 8; ++q) pk[u][ph][q] = pack8(v + 8 * q);
+                            }
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
+                    }
+                }
+                if (!alive) break;
+                #pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    #pragma unroll
+                    for (int ph = 0; ph < 2; ++ph)
+                        if (u < tc.nsub && (tc.tn + u) * TC_BN + ph * EPI_COLS < p.N) stage_and_store(pk[u][ph], (tc.tn + u) * TC_BN + ph * EPI_COLS);
+            } else
             for (int u = 0; u < tc.nsub && alive; ++u) {
                 const uint32_t acc = acc0 + u;
                 const int n0 = (tc.tn + u) * TC_BN;
@@ -670,30 +723,6 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     __syncwarp();
                     if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
                 };
-                if (!p.cin && !p.fuse_update && p.diag_add == 0.f) {
-                    // no axpy operand, no diagonal term (X' = B' X and X X^T): a thread's share of the accumulator fits in 64
-                    // packed registers, so read and pack all of it, release the accumulator, and only then stage and store.
-                    // For a macro-tile, whose epilogue nothing hides, this keeps the tensor cores' wait short.
-                    uint4 pk[2][8];
-                    #pragma unroll
-                    for (int ph = 0; ph < 2; ++ph) {
-                        if (ph < nphases) {
-                            float v[64];
-                            tmem_ld32(t_base + ph * EPI_COLS, v);
-                            tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
-                            tmem_ld_wait();
-                            #pragma unroll
-                            for (int j = 0; j < 64; ++j) v[j] *= c2;
-                            #pragma unroll
-                            for (int q = 0; q < 8; ++q) pk[ph][q] = pack8(v + 8 * q);
-                        }
-                    }
-                    release_acc();
-                    #pragma unroll
-                    for (int ph = 0; ph < 2; ++ph)
-                        if (ph < nphases) stage_and_store(pk[ph], n0 + ph * EPI_COLS);
-                    continue;
-                }
                 for (int ph = 0; ph < nphases; ++ph) {
                     float v[64];
                     tmem_ld32(t_base + ph * EPI_COLS, v);
