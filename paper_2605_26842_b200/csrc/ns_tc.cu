@@ -59,16 +59,22 @@ constexpr uint32_t B_SUB_BYTES = CTA_N * TC_BK * 2;               // 16 KiB per 
 constexpr int EPI_COLS = 128;                                     // output columns per epilogue phase
 constexpr uint32_t EPI_BUF_BYTES = CTA_M * EPI_COLS * 2;          // 32 KiB = 2 x 2 boxes: staging buffer of the store epilogue
 constexpr uint32_t TMEM_COLS = 512;                               // 2 accumulators x 256 fp32 columns
-constexpr int STAGES = 4;                                         // operand ring depth
-constexpr uint32_t STAGE_BYTES = A_STAGE_BYTES + 2 * B_SUB_BYTES; // 48 KiB: room for a macro-tile's k-slice
+// Operand staging: a ring of 16 KiB slabs.  A k-slice takes one slab per operand part it stages (1: diagonal tile whose
+// operands coincide, 2: plain tile, 3: macro-tile), contiguous (a k-slice that does not fit before the end of the ring
+// starts again at slab 0), so plain tiles run six k-slices ahead and macro-tiles four.  Every k-slice in flight owns one
+// entry of a ring of "full"/"empty" barriers; producer and MMA issuer derive the same slab positions from the item sequence.
+constexpr int NSLAB = 12;
+constexpr int NENT = 12;                                          // barrier entries = most k-slices in flight
+constexpr uint32_t SLAB_BYTES = 16384;
+static_assert(SLAB_BYTES == A_STAGE_BYTES && SLAB_BYTES == B_SUB_BYTES, "one slab per operand part");
 constexpr int RING = 4;                                           // published-but-unfinished work items
 constexpr uint32_t SMEM_CTRL_BYTES = 512;
-constexpr uint32_t SMEM_TOTAL = STAGES * STAGE_BYTES + EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
+constexpr uint32_t SMEM_TOTAL = NSLAB * SLAB_BYTES + EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
 constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
 // readers of a published item: producer + MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
 constexpr uint32_t RING_READERS = 2 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
 static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-static_assert(8 * (2 * STAGES + 4 + 2 * RING) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
+static_assert(8 * (2 * NENT + 4 + 2 * RING) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -348,11 +354,11 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const __grid_constant__ UpdateTable upd, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzle atoms need 1024-byte alignment
-    const uint32_t epi_buf = base + STAGES * STAGE_BYTES;
+    const uint32_t epi_buf = base + NSLAB * SLAB_BYTES;
     const uint32_t ctrl = epi_buf + EPI_BUF_BYTES;
-    const uint32_t bar_full = ctrl;                             // STAGES x 8 B (used in the leader)
-    const uint32_t bar_empty = bar_full + 8 * STAGES;           // STAGES x 8 B
-    const uint32_t bar_acc_full = bar_empty + 8 * STAGES;       // 2 x 8 B, one per accumulator
+    const uint32_t bar_full = ctrl;                             // NENT x 8 B (used in the leader)
+    const uint32_t bar_empty = bar_full + 8 * NENT;             // NENT x 8 B
+    const uint32_t bar_acc_full = bar_empty + 8 * NENT;         // 2 x 8 B, one per accumulator
     const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B (used in the leader)
     const uint32_t bar_ring_full = bar_acc_empty + 16;          // RING x 8 B
     const uint32_t bar_ring_empty = bar_ring_full + 8 * RING;   // RING x 8 B (used in the leader)
@@ -370,7 +376,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int q = 0; q < NS_MAX_PHASES; ++q) phase_items[q] = q < P ? (unsigned)g.ph[q].items_per_mat : 0u;
-        for (int s = 0; s < STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int s = 0; s < NENT; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -399,7 +405,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     };
 
     // TMA loads of all k-slices of one item into the stage ring (both CTAs run this, each for its own rows).
-    uint32_t stage = 0, phase = 0;
+    // producer's view of the slab ring: next entry, next slab, oldest entry not yet known to be free, free slabs, and
+    // the slabs every entry in flight took (3 bits each, wrap-around gap included)
+    uint32_t ent = 0, slab_head = 0, tail_ent = 0, slabs_free = NSLAB;
+    unsigned long long ent_cost = 0ull;
     const uint32_t full_leader = map_to_cta(bar_full, 0);
     auto produce = [&](const Item& it) -> bool {
         const NsPhase& p = g.ph[it.q];
@@ -420,12 +429,26 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         const int a_switch = p.a_sym ? (tc.tm + 1) * (TC_BM / TC_BK) : (p.a_mn ? 0 : num_kb);
         const int b_switch0 = p.b_sym ? (tc.tn + 1) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb);
         const int b_switch1 = p.b_sym ? (tc.tn + 2) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb);
+        const uint32_t nslab = 1u + (uint32_t)nb;
         for (int kb = 0; kb < num_kb; ++kb) {
-            if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 1)) return false;
-            const uint32_t full = full_leader + 8 * stage;
-            const uint32_t sa = base + stage * STAGE_BYTES;
+            const uint32_t gap = slab_head + nslab > NSLAB ? NSLAB - slab_head : 0u;     // slabs skipped at the end of the ring
+            const uint32_t need = gap + nslab;
+            while (slabs_free < need) {        // entries are released in order: take back the oldest one's slabs
+                const uint32_t e = tail_ent % NENT;
+                if (!mbar_wait(bar_empty + 8 * e, (tail_ent / NENT) & 1u, abort_flag, status, 1)) return false;
+                slabs_free += (uint32_t)(ent_cost >> (3 * e)) & 7u;
+                ++tail_ent;
+            }
+            slabs_free -= need;
+            const uint32_t e = ent % NENT;
+            ent_cost = (ent_cost & ~(7ull << (3 * e))) | ((unsigned long long)need << (3 * e));
+            const uint32_t pos = gap ? 0u : slab_head;
+            slab_head = pos + nslab == NSLAB ? 0u : pos + nslab;
+            ++ent;
+            const uint32_t full = full_leader + 8 * e;
+            const uint32_t sa = base + pos * SLAB_BYTES;
             const int k0 = kb * TC_BK;
-            if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * stage, tx_bytes);   // both CTAs' copies land here
+            if (rank == 0) mbar_arrive_expect_tx(bar_full + 8 * e, tx_bytes);   // both CTAs' copies land here
             if (kb >= a_switch) {
                 tma_load_3d(sa, a_box64, full, m0, k0, it.c);
                 tma_load_3d(sa + BOX_BYTES, a_box64, full, m0 + TC_BOX, k0, it.c);
@@ -449,7 +472,6 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                 }
             }
-            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         return true;
     };
@@ -467,16 +489,14 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 fence_proxy_async();       // the scheduler's acquire of the dependency precedes these copies
                 ok = produce(it);
             }
-            // stay until the tensor cores have released every stage: the commits arrive on this CTA's barriers
-            for (int s = 0; s < STAGES && ok; ++s) {
-                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, status, 5);
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-            }
+            // stay until the tensor cores have released every k-slice: the commits arrive on this CTA's barriers
+            for (; ok && tail_ent < ent; ++tail_ent)
+                ok = mbar_wait(bar_empty + 8 * (tail_ent % NENT), (tail_ent / NENT) & 1u, abort_flag, status, 5);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
-            uint32_t mstage = 0, mphase = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
+            uint32_t ment = 0, mslab = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
@@ -496,17 +516,21 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     b_switch[u] = shared_ab ? a_switch : (p.b_sym ? (tc.tn + u + 1) * (TC_BN / TC_BK) : (p.b_mn ? 0 : num_kb));
                 const uint32_t b_off0 = shared_ab ? 0u : (A_STAGE_BYTES >> 4);             // operand offsets inside a stage, in 16-byte units
                 const uint32_t b_off1 = (A_STAGE_BYTES + B_SUB_BYTES) >> 4;
-                // the accumulators must have been drained by the epilogue of their previous tile
-                for (int u = 0; u < tc.nsub && ok; ++u)
-                    ok = mbar_wait(bar_acc_empty + 8 * (acc0 + u), ((acc_par >> (acc0 + u)) & 1u) ^ 1u, abort_flag, status, 2);
-                if (!ok) break;
+                // an accumulator must have been drained by the epilogue of its previous tile before the first MMA into it
+                if (!(ok = mbar_wait(bar_acc_empty + 8 * acc0, ((acc_par >> acc0) & 1u) ^ 1u, abort_flag, status, 2))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + acc0 * TC_BN, d1 = d0 + TC_BN;
                 uint32_t accum = 0u;
-                uint32_t stage_lo = (base + mstage * STAGE_BYTES) >> 4;
+                const uint32_t nslab = shared_ab ? 1u : 1u + (uint32_t)tc.nsub;
                 for (int kb = 0; kb < num_kb; ++kb) {
+                    // same slab walk as the producer's
+                    const uint32_t pos = mslab + nslab > NSLAB ? 0u : mslab;
+                    mslab = pos + nslab == NSLAB ? 0u : pos + nslab;
+                    const uint32_t e = ment % NENT;
+                    const uint32_t stage_lo = (base + pos * SLAB_BYTES) >> 4;
                     // no tcgen05 fence here: the operands arrive through the asynchronous proxy and the barrier orders them
-                    if (!(ok = mbar_wait(bar_full + 8 * mstage, mphase, abort_flag, status, 3))) break;
+                    if (!(ok = mbar_wait(bar_full + 8 * e, (ment / NENT) & 1u, abort_flag, status, 3))) break;
+                    ++ment;
                     const uint32_t a_mn = kb >= a_switch ? 1u : 0u, b_mn0 = kb >= b_switch[0] ? 1u : 0u;
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
                     const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step0 = b_mn0 ? (2048u >> 4) : (32u >> 4);
@@ -519,6 +543,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         accum = 1u;
                     }
                     if (tc.nsub == 2) {
+                        if (kb == 0) {
+                            if (!(ok = mbar_wait(bar_acc_empty + 8 * (acc0 + 1), ((acc_par >> (acc0 + 1)) & 1u) ^ 1u, abort_flag, status, 2))) break;
+                            tc_fence_after();
+                        }
                         const uint32_t b_mn1 = kb >= b_switch[1] ? 1u : 0u;
                         const uint32_t b_step1 = b_mn1 ? (2048u >> 4) : (32u >> 4);
                         const uint32_t b_lo1 = (stage_lo + b_off1) | (b_mn1 ? DESC_LBO_MN : DESC_LBO_K);
@@ -528,9 +556,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         #pragma unroll
                         for (int k = 1; k < TC_BK / 16; ++k) tc_mma_bf16(d1, a_lo + k * a_step, b_lo1 + k * b_step1, idesc1, 1u);
                     }
-                    tc_commit_pair(bar_empty + 8 * mstage);     // frees the stage in both CTAs when these MMAs have read it
-                    stage_lo += STAGE_BYTES >> 4;
-                    if (++mstage == STAGES) { mstage = 0; mphase ^= 1u; stage_lo = base >> 4; }
+                    tc_commit_pair(bar_empty + 8 * e);     // frees the k-slice's slabs in both CTAs when these MMAs have read them
                 }
                 if (!ok) break;
                 for (int u = 0; u < tc.nsub; ++u) {
@@ -659,14 +685,14 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 // issuer as soon as it has been read, and only then stage and store.  Nothing hides the epilogue of a
                 // macro-tile, so the time the tensor cores wait is the time of these reads.
                 uint4 pk[2][2][8];
+                bool all_ok = true;
                 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     if (u < tc.nsub) {
                         const uint32_t acc = acc0 + u;
                         const int n0 = (tc.tn + u) * TC_BN;
-                        bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
-                        ok = epi_bar_all(3, ok);
-                        if (!ok) { alive = false; break; }
+                        // every warp goes ahead on its own; whether all of them got their data is agreed on after the reads
+                        if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { all_ok = false; break; }
                         tc_fence_after();
                         acc_par ^= 1u << acc;
                         const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
@@ -688,7 +714,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
                     }
                 }
-                if (!alive) break;
+                if (!epi_bar_all(3, all_ok)) { alive = false; break; }
                 #pragma unroll
                 for (int u = 0; u < 2; ++u)
                     #pragma unroll
