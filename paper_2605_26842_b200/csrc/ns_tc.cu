@@ -26,7 +26,9 @@
 //              memory and hand the boxes to TMA stores (a thread owns one row, so storing from registers
 //              would touch 32 lines per warp instruction; the TMA writes whole lines);
 //              for the last X' = B' X of a step the same warps apply the parameter update of Eq. muon_update
-//              to the fp32 weights instead.  When the item's stores have completed they count it as done.
+//              to the fp32 weights instead,
+//   warp 3     store warp: turns each staged phase into TMA stores, frees the staging buffer, and counts the item as
+//              done once its stores have completed, so that no epilogue warp ever waits for global memory.
 // Tensor memory holds two 256-column accumulators.  Plain tiles alternate between them, so the epilogue of one
 // tile overlaps the main loop of the next.  A macro-tile uses both at once, two neighbouring tiles computed
 // from ONE staged slice of the A operand: 96 KiB instead of 128 KiB cross from L2 per k-slice and pair.
@@ -42,7 +44,8 @@ namespace {
 
 constexpr int TC_EPI_WARPS = 8;                                   // two warps per tensor-memory lane quadrant
 constexpr int TC_EPI_THREADS = 32 * TC_EPI_WARPS;
-constexpr int SCHED_WARP = 2;                                     // the scheduler (leader CTA); warp 3 has no role
+constexpr int SCHED_WARP = 2;                                     // the scheduler (leader CTA)
+constexpr int STORE_WARP = 3;                                     // issues and retires the TMA stores of the epilogue
 constexpr int EPI_WARP0 = 4;                                      // epilogue = warps 4..11, i.e. warpgroups 1 and 2
 constexpr int TC_THREADS = 32 * EPI_WARP0 + TC_EPI_THREADS;       // 384
 // The kernel starts with 168 registers per thread (12 warps x 32 x 168 fit the SM's 64 K); then the warpgroup of the
@@ -71,10 +74,11 @@ constexpr int RING = 4;                                           // published-b
 constexpr uint32_t SMEM_CTRL_BYTES = 512;
 constexpr uint32_t SMEM_TOTAL = NSLAB * SLAB_BYTES + EPI_BUF_BYTES + SMEM_CTRL_BYTES + 1024;
 constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
-// readers of a published item: producer + MMA issuer + epilogue warps in the leader, producer + epilogue warps in the peer
-constexpr uint32_t RING_READERS = 2 + TC_EPI_WARPS + 1 + TC_EPI_WARPS;
+// readers of a published item: producer, MMA issuer, store warp and epilogue warps in the leader; producer, store warp and
+// epilogue warps in the peer
+constexpr uint32_t RING_READERS = 3 + TC_EPI_WARPS + 2 + TC_EPI_WARPS;
 static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-static_assert(8 * (2 * NENT + 4 + 2 * RING) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
+static_assert(8 * (2 * NENT + 4 + 2 * RING + 2) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -106,6 +110,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 // Arrive (release at cluster scope) on a barrier given by its cluster-wide address (own CTA or the peer).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // The same with the default semantics, for hand-overs that carry no shared-memory data (tensor-memory accumulators).
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
@@ -180,24 +187,6 @@ __device__ __forceinline__ bool wait_counter(const unsigned int* ctr, unsigned n
             }
         }
     }
-}
-
-// ---- named barriers among the epilogue warps ------------------------------------------------------
-__device__ __forceinline__ void epi_bar_sync(int id) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(TC_EPI_THREADS) : "memory");
-}
-// Barrier + AND-reduction of a predicate over the epilogue threads (same answer in every thread).
-__device__ __forceinline__ bool epi_bar_all(int id, bool pred) {
-    uint32_t in = pred ? 1u : 0u, out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "barrier.cta.red.and.pred p, %2, %3, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out)
-        : "r"(in), "r"(id), "r"(TC_EPI_THREADS)
-        : "memory");
-    return out != 0;
 }
 
 // ---- TMA ------------------------------------------------------------------------------------------
@@ -362,7 +351,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B (used in the leader)
     const uint32_t bar_ring_full = bar_acc_empty + 16;          // RING x 8 B
     const uint32_t bar_ring_empty = bar_ring_full + 8 * RING;   // RING x 8 B (used in the leader)
-    const uint32_t tmem_slot = bar_ring_empty + 8 * RING;       // 4 B + abort flag 4 B + 8 B pad
+    const uint32_t bar_stg_full = bar_ring_empty + 8 * RING;    // staging buffer written (one arrival per epilogue warp)
+    const uint32_t bar_stg_empty = bar_stg_full + 8;            // staging buffer read by the stores (store warp)
+    const uint32_t tmem_slot = bar_stg_empty + 8;               // 4 B + abort flag 4 B + 8 B pad
     const uint32_t ring_items = tmem_slot + 16;                 // RING x 16 B
     volatile unsigned int* phase_items = reinterpret_cast<volatile unsigned int*>(smem_raw + (ring_items + 16 * RING - smem_u32(smem_raw)));   // NS_MAX_PHASES x 4 B
     uint8_t* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
@@ -379,6 +370,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         for (int s = 0; s < NENT; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
+        mbar_init(bar_stg_full, TC_EPI_WARPS);
+        mbar_init(bar_stg_empty, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         #pragma unroll
         for (int i = 0; i < NS_MAPS; ++i) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[i]) : "memory");
@@ -567,6 +560,47 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 if (tc.nsub == 1) acc_next ^= 1u;
             }
         }
+    } else if (warp == STORE_WARP) {
+        if (lane == 0) {
+            // ---------------- store warp (both CTAs) ----------------
+            // Sends every staged phase of the epilogue to D with TMA stores (this thread owns the bulk-copy groups, so it is
+            // the one that can wait for them), frees the staging buffer when a phase has been read, and counts the item as
+            // done for its matrix and phase once all of its stores have completed.  The epilogue warps never wait for global
+            // memory.  It walks the items and their phases in the epilogue's order.
+            uint32_t staged = 0;
+            bool ok = true;
+            for (unsigned n = 0; ok; ++n) {
+                Item it;
+                if (!(ok = take_item(n, it, 12, true)) || it.stop) break;
+                const NsPhase& p = g.ph[it.q];
+                if (p.fuse_update) continue;               // the epilogue writes the parameters itself; nothing is staged
+                const CUtensorMap* tma_d = &maps.m[p.d_map + NS_TENSORS];     // 64 columns x 128 rows per store
+                const TileCoord tc = decode_tile(p, it.t);
+                const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
+                for (int u = 0; u < tc.nsub && ok; ++u) {
+                    for (int ph = 0; ph < 2 && ok; ++ph) {
+                        const int x0 = (tc.tn + u) * TC_BN + ph * EPI_COLS;
+                        if (x0 >= p.N) continue;
+                        if (!(ok = mbar_wait(bar_stg_full, staged & 1u, abort_flag, status, 13))) break;
+                        ++staged;
+                        #pragma unroll
+                        for (int bx = 0; bx < 2; ++bx) {
+                            const int x = x0 + bx * TC_BOX;
+                            if (x < p.N && m0 < p.M) tma_store_3d(tma_d, epi_buf + bx * 2 * BOX_BYTES, x, m0, it.c);   // clipped at the extents
+                        }
+                        bulk_commit();
+                        bulk_wait_read();                  // the stores have read the buffer: the epilogue may refill it
+                        mbar_arrive_local(bar_stg_empty);
+                    }
+                }
+                if (!ok) break;
+                bulk_wait_all();                           // the item's output is in global memory
+                fence_proxy_async();
+                __threadfence();
+                atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
+            }
+            bulk_wait_all();           // shared memory must outlive the stores that read it
+        }
     } else if (warp == SCHED_WARP) {
         if (lane == 0 && rank == 0) {
             // ---------------- scheduler (leader CTA only) ----------------
@@ -629,27 +663,39 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         // A warp may only read the 32 tensor-memory lanes of its quadrant (warp index mod 4).  A 256-column
         // tile is handled in phases of 128 columns; in a phase the two warps of a quadrant take 64 columns
         // each, so a thread owns 64 consecutive columns of one row: one 128-byte line of the bf16 output.
+        // The warps run independently of one another: they meet only at the staging buffer's two barriers.
         const int quad = warp & 3;
         const int half = (warp - EPI_WARP0) >> 2;
         const int row_in_cta = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const uint32_t acc_empty_leader = map_to_cta(bar_acc_empty, 0);
-        const bool issuer = threadIdx.x == 32 * EPI_WARP0;     // first epilogue thread: issues and retires TMA stores
         // position of this thread's row inside the staging buffer: one 128-row box per column half, 128-byte rows
         const uint32_t stage_off = (uint32_t)half * (2u * BOX_BYTES) + (uint32_t)row_in_cta * 128u;
         const uint32_t swz = (uint32_t)row_in_cta & 7u;
         uint32_t acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
+        uint32_t staged = 0;                  // staging phases handed to the store warp so far
         bool alive = true;
+        // 128 packed columns of this thread's row go to the staging buffer; the store warp sends them on
+        auto put_phase = [&](const uint4* pk) -> bool {
+            if (!mbar_wait(bar_stg_empty, (staged & 1u) ^ 1u, abort_flag, status, 11)) return false;   // the previous phase has been read
+            #pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t addr = epi_buf + stage_off + (((uint32_t)q ^ swz) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q].x), "r"(pk[q].y), "r"(pk[q].z), "r"(pk[q].w) : "memory");
+            }
+            fence_proxy_async();                   // generic-proxy writes above must be visible to the TMA engine
+            __syncwarp();
+            if (lane == 0) mbar_arrive_local(bar_stg_full);
+            ++staged;
+            return true;
+        };
         for (unsigned n = 0; alive; ++n) {
             Item it;
-            bool got = take_item(n, it, 10, false);
-            got = epi_bar_all(3, got);         // all epilogue threads take the same exit, so no one is left at a barrier
-            if (!got) break;
+            if (!take_item(n, it, 10, false)) break;
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(ring_empty_leader + 8 * (n % RING));   // every lane has its copy of the item
             if (it.stop) break;
             const NsPhase& p = g.ph[it.q];
-            const CUtensorMap* tma_d = &maps.m[p.d_map + NS_TENSORS];     // 64 columns x 128 rows per store
             const TileCoord tc = decode_tile(p, it.t);
             const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
             const int gr = m0 + row_in_cta;
@@ -659,40 +705,18 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             if (p.post_mode) { const float sc = g.inv_norm[it.c]; post = p.post_mode == 2 ? sc * sc : sc; }
             const float c1 = p.c1 * post, c2 = p.c2 * post;
             const uint32_t acc0 = tc.nsub == 2 ? 0u : acc_next;
-            // 128 packed columns of this thread's row go to the staging buffer and from there, as four boxes, to D
-            auto stage_and_store = [&](const uint4* pk, int x0) {
-                if (issuer) bulk_wait_read();          // the stores issued for the previous phase have read the buffer
-                epi_bar_sync(1);
-                #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const uint32_t addr = epi_buf + stage_off + (((uint32_t)q ^ swz) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q].x), "r"(pk[q].y), "r"(pk[q].z), "r"(pk[q].w) : "memory");
-                }
-                fence_proxy_async();                   // generic-proxy writes above must be visible to the TMA engine
-                epi_bar_sync(2);
-                if (issuer) {
-                    #pragma unroll
-                    for (int bx = 0; bx < 2; ++bx) {
-                        const int x = x0 + bx * TC_BOX;
-                        if (x < p.N && m0 < p.M) tma_store_3d(tma_d, epi_buf + bx * 2 * BOX_BYTES, x, m0, it.c);   // clipped at the extents
-                    }
-                    bulk_commit();
-                }
-            };
             if (!p.cin && !p.fuse_update && p.diag_add == 0.f) {
                 // No axpy operand, no diagonal term (X X^T and X' = B' X).  A thread's share of an accumulator is 128 values,
                 // 64 registers once packed: read and pack every accumulator of the item first, handing each back to the MMA
-                // issuer as soon as it has been read, and only then stage and store.  Nothing hides the epilogue of a
-                // macro-tile, so the time the tensor cores wait is the time of these reads.
+                // issuer as soon as it has been read, and only then stage.  Nothing hides the epilogue of a macro-tile, so
+                // the time the tensor cores wait is the time of these reads.
                 uint4 pk[2][2][8];
-                bool all_ok = true;
                 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    if (u < tc.nsub) {
+                    if (u < tc.nsub && alive) {
                         const uint32_t acc = acc0 + u;
                         const int n0 = (tc.tn + u) * TC_BN;
-                        // every warp goes ahead on its own; whether all of them got their data is agreed on after the reads
-                        if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { all_ok = false; break; }
+                        if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { alive = false; break; }
                         tc_fence_after();
                         acc_par ^= 1u << acc;
                         const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
@@ -714,12 +738,11 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
                     }
                 }
-                if (!epi_bar_all(3, all_ok)) { alive = false; break; }
                 #pragma unroll
                 for (int u = 0; u < 2; ++u)
                     #pragma unroll
                     for (int ph = 0; ph < 2; ++ph)
-                        if (u < tc.nsub && (tc.tn + u) * TC_BN + ph * EPI_COLS < p.N) stage_and_store(pk[u][ph], (tc.tn + u) * TC_BN + ph * EPI_COLS);
+                        if (alive && u < tc.nsub && (tc.tn + u) * TC_BN + ph * EPI_COLS < p.N) alive = put_phase(pk[u][ph]);
             } else
             for (int u = 0; u < tc.nsub && alive; ++u) {
                 const uint32_t acc = acc0 + u;
@@ -737,24 +760,21 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                 };
                 if (p.cin) load_cin(0);
-                bool ok = mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4);
-                ok = epi_bar_all(3, ok);
-                if (!ok) { alive = false; break; }
+                if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { alive = false; break; }
                 tc_fence_after();
                 acc_par ^= 1u << acc;
                 const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
-                auto release_acc = [&]() {
-                    // this warp has read all it needs from the accumulator: hand it back to the MMA issuer
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
-                };
-                for (int ph = 0; ph < nphases; ++ph) {
+                for (int ph = 0; ph < nphases && alive; ++ph) {
                     float v[64];
                     tmem_ld32(t_base + ph * EPI_COLS, v);
                     tmem_ld32(t_base + ph * EPI_COLS + 32, v + 32);
                     tmem_ld_wait();
-                    if (ph == nphases - 1) release_acc();
+                    if (ph == nphases - 1) {
+                        // this warp has read all it needs from the accumulator: hand it back to the MMA issuer
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_remote(acc_empty_leader + 8 * acc);
+                    }
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
                     if (p.cin) {
                         const uint32_t w[32] = {cin_raw[0].x, cin_raw[0].y, cin_raw[0].z, cin_raw[0].w, cin_raw[1].x, cin_raw[1].y,
@@ -781,9 +801,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         uint4 pk[8];
                         #pragma unroll
                         for (int q = 0; q < 8; ++q) pk[q] = pack8(v + 8 * q);
-                        stage_and_store(pk, n0 + ph * EPI_COLS);
+                        alive = put_phase(pk);
                     } else if (row_ok) {
-                        // Eq. muon_update on this thread's 64 parameters: W <- (W - eta lambda W) - eta gamma O
+                        // Eq. muon_update on this thread's 64 parameters: W <- (W - eta lambda W) - eta gamma O.  Nothing in the
+                        // launch reads these stores (the phase is the last one of the step), so they need no completion signal.
                         float* wrow = upd.w[it.c] + (long long)gr * p.ld + gc0;
                         float* orow = upd.o[it.c] ? upd.o[it.c] + (long long)gr * p.ld + gc0 : nullptr;
                         #pragma unroll
@@ -800,20 +821,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                 }
             }
-            if (!alive) break;
             if (tc.nsub == 1) acc_next ^= 1u;
-            // count the item as done for its matrix and phase once its output is in global memory: the TMA stores have
-            // completed (issuer) and every thread's own stores are fenced; then one arrival per CTA
-            if (issuer) bulk_wait_all();
-            fence_proxy_async();
-            __threadfence();
-            epi_bar_sync(1);
-            if (issuer) {
-                __threadfence();
-                atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
-            }
         }
-        if (issuer) bulk_wait_all();           // shared memory must outlive the stores that read it
     }
 
     if (*abort_flag) __nanosleep(200000);      // let copies that are still in flight land before the CTA goes away
