@@ -122,12 +122,14 @@ mona_status mona_default_hparams(mona_hparams* hp);
  *                        that the start and the tail of one chunk's kernels are filled by the other chunk's;
  *                        0 keeps every launch on the caller's stream.  Results are identical either way; the
  *                        workspace holds two chunks.
- *   fuse_update        : 1 (default): on the tensor-core path the last X' = B' X of a step applies Eq. muon_update
- *                        in its epilogue (fp32 O_k straight from the accumulator, no bf16 copy of O_k written and
- *                        re-read, no separate update kernel).  0: O_k is stored in bf16 and a separate elementwise
- *                        kernel updates the parameters.  The two differ by the bf16 rounding of O_k only.
+ *   fuse_update        : 0 (default): O_k is stored in bf16 and a separate elementwise kernel applies Eq. muon_update.
+ *                        1: on the tensor-core path the last X' = B' X of a step applies the update in its epilogue
+ *                        (fp32 O_k straight from the accumulator, no bf16 copy of O_k written and re-read, one launch
+ *                        fewer per chunk).  The two differ by the bf16 rounding of O_k only.  Measured slower on the
+ *                        benchmark sets: a thread owns a row of the accumulator, so its fp32 read-modify-write of W
+ *                        touches 32 lines per warp instruction and sits, unhidden, in the macro-tile's epilogue.
  *   ns_delay           : how many matrices apart consecutive Newton-Schulz GEMMs of one matrix sit in the kernel's
- *                        work order (0 = the default, 3; at most 1024; a value >= the chunk's matrix count
+ *                        work order (0 = the default, 6; at most 1024; a value >= the chunk's matrix count
  *                        runs the chunk GEMM by GEMM).  Larger values hide the dependency latency
  *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it. */
 typedef struct {

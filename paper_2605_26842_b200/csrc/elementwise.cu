@@ -9,7 +9,9 @@ namespace mona {
 
 namespace {
 
-constexpr int EW_THREADS = 256;
+// 128-thread blocks of ~46 registers: small enough to run on an SM beside a resident CTA of the Newton-Schulz kernel
+// (which leaves 7168 registers free), so the elementwise passes of one chunk overlap the GEMMs of another.
+constexpr int EW_THREADS = 128;
 
 __device__ __forceinline__ float mul_add2(F2 k, float x, float addend) {
     // (k.hi + k.lo) * x + addend with a single rounding on the dominant term

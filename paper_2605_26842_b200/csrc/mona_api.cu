@@ -251,8 +251,8 @@ mona_status mona_default_options(mona_options* opt) {
     memset(opt, 0, sizeof *opt);
     opt->chunk_budget_bytes = g_chunk_budget_bytes.load();
     opt->chunk_overlap = g_chunk_overlap.load();
-    opt->fuse_update = 1;
-    opt->ns_delay = 3;
+    opt->fuse_update = 0;
+    opt->ns_delay = 6;
     return MONA_OK;
 }
 

@@ -48,12 +48,15 @@ constexpr int SCHED_WARP = 2;                                     // the schedul
 constexpr int STORE_WARP = 3;                                     // issues and retires the TMA stores of the epilogue
 constexpr int EPI_WARP0 = 4;                                      // epilogue = warps 4..11, i.e. warpgroups 1 and 2
 constexpr int TC_THREADS = 32 * EPI_WARP0 + TC_EPI_THREADS;       // 384
-// The kernel starts with 168 registers per thread (12 warps x 32 x 168 fit the SM's 64 K); then the warpgroup of the
-// producer, MMA issuer and scheduler gives registers back and the two epilogue warpgroups take them (setmaxnreg):
-// 128 x 48 + 256 x 224 = 63488.  An epilogue thread can then hold its share of BOTH accumulators of a macro-tile.
-constexpr int TC_MAX_REGS = 168;
-constexpr int REGS_CONTROL = 48;
-constexpr int REGS_EPILOGUE = 224;
+// The kernel starts with 152 registers per thread (12 warps x 32 x 152 = 58368 of the SM's 65536: the rest, together
+// with the ~1.5 KiB of shared memory the kernel leaves, lets one 128-thread block of the elementwise kernels of the
+// NEXT chunk run beside it, so prologue and update overlap the GEMMs instead of waiting for the SMs).  Then the
+// warpgroup of the producer, MMA issuer, scheduler and store warp gives registers back and the two epilogue warpgroups
+// take them (setmaxnreg): 128 x 40 + 256 x 208 = 58368.  An epilogue thread can then hold its share of BOTH
+// accumulators of a macro-tile.
+constexpr int TC_MAX_REGS = 152;
+constexpr int REGS_CONTROL = 40;
+constexpr int REGS_EPILOGUE = 208;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
 constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
@@ -338,7 +341,7 @@ struct UpdateTable {
     float* o[MAXC];
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(TC_MAX_REGS)
 ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsProgram g,
                 const __grid_constant__ UpdateTable upd, DeviceStatus* __restrict__ status) {
     extern __shared__ uint8_t smem_raw[];

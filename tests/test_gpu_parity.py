@@ -63,12 +63,12 @@ def test_mixed_set_ten_steps():
     check(errs, TOL_O_BF16)
 
 
-def test_separate_update_kernel_matches_too():
-    """fuse_update = 0: O_k stored in bf16 and a separate elementwise kernel applies Eq. muon_update."""
+def test_update_fused_into_the_last_gemm_matches_too():
+    """fuse_update = 1: the last X' = B' X applies Eq. muon_update in its epilogue (fp32 O_k from the accumulator)."""
     shapes = [(3, 256, 512), (2, 512, 256), (1, 320, 192)]
-    errs = run_case(shapes, steps=3, seed=43, options=pkg.default_options(fuse_update=0))
+    errs = run_case(shapes, steps=3, seed=43, options=pkg.default_options(fuse_update=1))
     check(errs, TOL_O_BF16)
-    assert errs["launches"] == 3 * 3        # per chunk: prologue, Newton-Schulz, update
+    assert errs["launches"] == 3 * 2        # per chunk: prologue, Newton-Schulz (update inside)
 
 
 @pytest.mark.parametrize("delay", [1, 2, 7])
