@@ -29,12 +29,12 @@ if ROOT not in sys.path:
 METRIC = "mona_optimizer_steps_per_s"
 UNIT = "steps/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the GEMM kernel from the ncu capture
-# summarised in profiles/tc_gemm_kernel_moe7b_768x2048_per_launch.md: mean over the 15 launches of one 93-matrix
-# 768x2048 chunk, the launch shape that makes up most of the default workload.  Valid only for the kernel source
-# the counters were taken with (hash of ns_tc.cu + ns_tc.cuh).
-NCU_TRAFFIC = {"source_sha256_16": "553d71a096c0df77", "bytes_per_launch": 357.1e6,
-               "unit": "DRAM bytes per launch (ncu, 93-matrix 768x2048 chunk)"}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the Newton-Schulz kernel from the ncu capture
+# summarised in profiles/ns_chunk_kernel_moe7b_1L.md: the launch over a 93-matrix 768x2048 chunk, the launch shape that
+# makes up most of the default workload (40 of its 56 launches per step are of this shape or its tall twin).  Valid only
+# for the kernel source the counters were taken with (hash of ns_tc.cu + ns_tc.cuh).
+NCU_TRAFFIC = {"source_sha256_16": "1757ceb5f34864a9", "bytes_per_launch": 6.081e9,
+               "unit": "DRAM bytes of one launch over a 93-matrix 768x2048 chunk (ncu; 2.153 TFLOP executed in that launch)"}
 
 
 def kernel_traffic():
