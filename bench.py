@@ -244,6 +244,8 @@ def run_workload(torch, pkg, synth, shard, args, dev, local_rank, rank, world, d
         options.fuse_update = 1
     if args.ns_delay:
         options.ns_delay = args.ns_delay
+    if args.macro_min_k:
+        options.macro_tile_min_k = args.macro_min_k
     # every rank owns an independent parameter set of this shape (weak scaling, no data-path collective)
     params = synth.init_params(wl, dev, seed_offset=rank)
     gp = synth.GradientProcess(wl, dev, keep_fp32_shadow=False)
@@ -447,6 +449,7 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="keep all chunks on one stream")
     ap.add_argument("--fuse", action="store_true", help="apply the parameter update in the epilogue of the last GEMM instead of a separate kernel")
     ap.add_argument("--ns-delay", type=int, default=None, help="work-order distance between consecutive GEMMs of one matrix")
+    ap.add_argument("--macro-min-k", type=int, default=None, help="shortest inner dimension for which X' = B'X uses 256x512 macro-tiles")
     ap.add_argument("--shard", action="store_true", help="one parameter set partitioned over the ranks, parameters exchanged after the step")
     ap.add_argument("--muon", action="store_true", help="plain Muon step (no acceleration term): the baseline of the paper's timing claim")
     ap.add_argument("--single-buffer", action="store_true", help="state kept as M and Z = beta_a A - (1 - beta_a) G (one fp32 buffer instead of A and G_prev)")

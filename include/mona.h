@@ -50,7 +50,8 @@ typedef enum {
     MONA_ERR_TIMEOUT = 5,            /* a bounded device-side wait ran out                            */
     MONA_ERR_NONFINITE = 6,          /* ||M_k||_F of some matrix was inf/nan                          */
     MONA_ERR_ARCH = 7,               /* device is not compute capability 10.x                         */
-    MONA_ERR_BUFFER_TOO_SMALL = 8    /* state or workspace smaller than mona_query_sizes() reports    */
+    MONA_ERR_BUFFER_TOO_SMALL = 8,   /* state or workspace smaller than mona_query_sizes() reports    */
+    MONA_ERR_BOUNDS = 9              /* debug build (-DMONA_DEBUG) only: a kernel's index check failed */
 } mona_status;
 
 typedef enum { MONA_F32 = 0, MONA_BF16 = 1 } mona_dtype;
@@ -131,13 +132,21 @@ mona_status mona_default_hparams(mona_hparams* hp);
  *   ns_delay           : how many matrices apart consecutive Newton-Schulz GEMMs of one matrix sit in the kernel's
  *                        work order (0 = the default, 6; at most 1024; a value >= the chunk's matrix count
  *                        runs the chunk GEMM by GEMM).  Larger values hide the dependency latency
- *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it. */
+ *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it.
+ *   macro_tile_min_k   : X' = B' X runs as 256 x 512 macro-tiles (two tiles sharing one staged operand slice, both
+ *                        accumulators in use, so nothing hides their epilogue) when its inner dimension - the shorter
+ *                        side of the weight - is at least this, and as plain 256 x 256 tiles with alternating
+ *                        accumulators below it (0 = the default, 1: always macro-tiles.  Plain tiles keep the tensor
+ *                        cores busier per clock on short inner dimensions, but the step runs at the power cap and
+ *                        macro-tiles move fewer bytes per flop: measured 3-7 % faster on every benchmark set).
+ *                        Results do not depend on it. */
 typedef struct {
     size_t chunk_budget_bytes;
     int32_t chunk_overlap;
     int32_t fuse_update;
     int32_t ns_delay;
-    int32_t reserved[5];       /* zero */
+    int32_t macro_tile_min_k;
+    int32_t reserved[4];       /* zero */
 } mona_options;
 
 /* Fills *opt with the defaults (as changed by the two process-wide setters below, if they were called). */

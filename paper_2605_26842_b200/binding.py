@@ -8,11 +8,12 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libmona.so")
+# MONA_LIBRARY selects another build of the same library (e.g. libmona_debug.so, the -DMONA_DEBUG build with index checks)
+_LIB_PATH = os.environ.get("MONA_LIBRARY") or os.path.join(_HERE, "libmona.so")
 
 STATUS_NAMES = {0: "MONA_OK", 1: "MONA_ERR_INVALID_ARG", 2: "MONA_ERR_UNSUPPORTED_SHAPE", 3: "MONA_ERR_ALIGNMENT",
                 4: "MONA_ERR_CUDA", 5: "MONA_ERR_TIMEOUT", 6: "MONA_ERR_NONFINITE", 7: "MONA_ERR_ARCH",
-                8: "MONA_ERR_BUFFER_TOO_SMALL"}
+                8: "MONA_ERR_BUFFER_TOO_SMALL", 9: "MONA_ERR_BOUNDS"}
 MONA_F32, MONA_BF16 = 0, 1
 MONA_STATE_COMBINED = 2      # single auxiliary buffer Z = beta_a A - (1 - beta_a) G
 
@@ -38,7 +39,7 @@ class Hparams(C.Structure):
 class Options(C.Structure):
     """mona_options: per-handle tuning knobs (see include/mona.h)."""
     _fields_ = [("chunk_budget_bytes", C.c_size_t), ("chunk_overlap", C.c_int32), ("fuse_update", C.c_int32),
-                ("ns_delay", C.c_int32), ("reserved", C.c_int32 * 5)]
+                ("ns_delay", C.c_int32), ("macro_tile_min_k", C.c_int32), ("reserved", C.c_int32 * 4)]
 
 
 _lib = None

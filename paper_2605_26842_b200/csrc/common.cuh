@@ -40,6 +40,17 @@ struct DeviceStatus {
 };
 constexpr unsigned STATUS_NONFINITE = 1u;
 constexpr unsigned STATUS_TIMEOUT = 2u;
+constexpr unsigned STATUS_BOUNDS = 4u;       // debug build only: an index check failed (site in timeout_site)
+
+// Index checks of the debug build (-DMONA_DEBUG).  compute-sanitizer is not available everywhere this library is
+// developed, so the kernels can check their own indices: a failed check latches STATUS_BOUNDS with a site number in the
+// status word - it never traps - and the guarded access is skipped.  In the normal build the macro is `true`.
+#ifdef MONA_DEBUG
+#define MONA_IN_BOUNDS(cond, status, site) \
+    ((cond) ? true : (atomicOr(&(status)->flags, ::mona::STATUS_BOUNDS), (status)->timeout_site = (site), false))
+#else
+#define MONA_IN_BOUNDS(cond, status, site) true
+#endif
 
 // A scalar hyper-parameter carried as an unevaluated sum of two floats, hi + lo, so that products with
 // it are accurate to ~2^-45 instead of 2^-24: rounding beta_a = 0.99 to one float would by itself

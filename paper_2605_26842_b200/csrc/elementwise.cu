@@ -164,6 +164,7 @@ prologue_kernel(ChunkPtrs ptrs, float* __restrict__ Mst, void* __restrict__ Ast,
     const int c = blockIdx.y, p = blockIdx.x;
     const long long lo = (long long)p * slab_len;
     const long long hi = (lo + slab_len < e) ? lo + slab_len : e;
+    if (!MONA_IN_BOUNDS(c < MAXC && p < slabs && p < MAX_SLABS && lo < e && (VEC == 1 || (lo % 4 == 0 && e % 4 == 0)), status, 201)) return;
     const GT* __restrict__ g = reinterpret_cast<const GT*>(ptrs.g[c]);
     float* __restrict__ M = Mst + (long long)c * e;
     using AuxT = typename StateIO<ST>::elem;

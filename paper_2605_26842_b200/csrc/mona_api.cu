@@ -253,6 +253,7 @@ mona_status mona_default_options(mona_options* opt) {
     opt->chunk_overlap = g_chunk_overlap.load();
     opt->fuse_update = 0;
     opt->ns_delay = 6;
+    opt->macro_tile_min_k = 1;
     return MONA_OK;
 }
 
@@ -271,6 +272,8 @@ mona_status resolve_options(const mona_options* in, mona_options& out) {
     out.fuse_update = in->fuse_update ? 1 : 0;
     if (in->ns_delay < 0 || in->ns_delay > 1024) return MONA_ERR_INVALID_ARG;
     if (in->ns_delay > 0) out.ns_delay = in->ns_delay;
+    if (in->macro_tile_min_k < 0) return MONA_ERR_INVALID_ARG;
+    if (in->macro_tile_min_k > 0) out.macro_tile_min_k = in->macro_tile_min_k;
     return MONA_OK;
 }
 }  // namespace
@@ -493,8 +496,8 @@ static mona_status step_impl(mona_handle* h, const mona_hparams* hp, void* const
                             g2.M = g2.N = g2.K = (int)b.s; g2.a_map = g2.b_map = MAP_A; g2.a_sym = g2.b_sym = 1; g2.symmetric = 1; g2.ab_same = 1;
                             g2.cin = ab; g2.d_map = MAP_B; g2.ld = b.s; g2.mat_stride = b.s * b.s; g2.c1 = ns_b; g2.c2 = ns_c; g2.diag_add = ns_a;
                             ns_phase_plan(g2);
-                            NsPhase& g3 = g.ph[3 * (t - t0) + 2];  // X' = B' X (wide) or X B' (tall), 256 x 512 macro-tiles
-                            g3.K = (int)b.s; g3.wide = 1; g3.d_map = MAP_X0 + nxt; g3.ld = b.cols; g3.mat_stride = b.e;
+                            NsPhase& g3 = g.ph[3 * (t - t0) + 2];  // X' = B' X (wide) or X B' (tall); 256 x 512 macro-tiles when the inner dimension is long
+                            g3.K = (int)b.s; g3.wide = b.s >= h->opt.macro_tile_min_k ? 1 : 0; g3.d_map = MAP_X0 + nxt; g3.ld = b.cols; g3.mat_stride = b.e;
                             g3.c1 = 0.f; g3.c2 = 1.f; g3.post_mode = t == 0 ? 1 : 0;
                             g3.fuse_update = (update_fused && t == T - 1) ? 1 : 0;
                             if (!b.tall) {   // B' is the symmetric "A" operand, X the MN-major "B" operand
@@ -684,6 +687,7 @@ mona_status mona_poll_status(mona_handle* h, void* stream_v, int64_t* first_bad_
     MONA_CUDA(h, cudaStreamSynchronize(stream));
     const DeviceStatus s = *h->host_status;
     if (first_bad_matrix) *first_bad_matrix = (s.first_bad == INT_MAX) ? -1 : s.first_bad;
+    if (s.flags & STATUS_BOUNDS) return h->fail(MONA_ERR_BOUNDS, "an index check of the debug build failed (site %u)", s.timeout_site);
     if (s.flags & STATUS_TIMEOUT) return h->fail(MONA_ERR_TIMEOUT, "a device-side wait ran out (site %u)", s.timeout_site);
     if (s.flags & STATUS_NONFINITE) return h->fail(MONA_ERR_NONFINITE, "non-finite ||M||_F, first at matrix %d", s.first_bad);
     return MONA_OK;

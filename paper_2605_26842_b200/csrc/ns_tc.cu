@@ -441,6 +441,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             const uint32_t pos = gap ? 0u : slab_head;
             slab_head = pos + nslab == NSLAB ? 0u : pos + nslab;
             ++ent;
+            if (!MONA_IN_BOUNDS(pos + nslab <= NSLAB && e < NENT && it.c < g.C, status, 102)) return false;
             const uint32_t full = full_leader + 8 * e;
             const uint32_t sa = base + pos * SLAB_BYTES;
             const int k0 = kb * TC_BK;
@@ -523,6 +524,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     const uint32_t pos = mslab + nslab > NSLAB ? 0u : mslab;
                     mslab = pos + nslab == NSLAB ? 0u : pos + nslab;
                     const uint32_t e = ment % NENT;
+                    if (!MONA_IN_BOUNDS(pos + nslab <= NSLAB && tc.tm < p.tiles_m && tc.tn + tc.nsub <= p.tiles_n, status, 103)) { ok = false; break; }
                     const uint32_t stage_lo = (base + pos * SLAB_BYTES) >> 4;
                     // no tcgen05 fence here: the operands arrive through the asynchronous proxy and the barrier orders them
                     if (!(ok = mbar_wait(bar_full + 8 * e, (ment / NENT) & 1u, abort_flag, status, 3))) break;
@@ -584,6 +586,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     for (int ph = 0; ph < 2 && ok; ++ph) {
                         const int x0 = (tc.tn + u) * TC_BN + ph * EPI_COLS;
                         if (x0 >= p.N) continue;
+                        if (!MONA_IN_BOUNDS(m0 < p.M + CTA_M && it.c < g.C && tc.tm < p.tiles_m, status, 106)) { ok = false; break; }
                         if (!(ok = mbar_wait(bar_stg_full, staged & 1u, abort_flag, status, 13))) break;
                         ++staged;
                         #pragma unroll
@@ -646,6 +649,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const unsigned idx = atomicAdd(g.work_counter, 1u);
                 Item it;
                 decode(idx, it);
+                if (!it.stop && !MONA_IN_BOUNDS(it.c >= 0 && it.c < g.C && it.q >= 0 && it.q < P && it.t >= 0 && (unsigned)it.t < phase_items[it.q], status, 101)) {
+                    latch_timeout(abort_flag, status, 101);        // an item that does not exist: give up the launch, cleanly
+                    break;
+                }
                 const unsigned int* ctr; unsigned need;
                 dependency(it, ctr, need);
                 if (ctr && !(ok = wait_counter(ctr, need, abort_flag, status, 6))) break;
@@ -681,6 +688,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         // 128 packed columns of this thread's row go to the staging buffer; the store warp sends them on
         auto put_phase = [&](const uint4* pk) -> bool {
             if (!mbar_wait(bar_stg_empty, (staged & 1u) ^ 1u, abort_flag, status, 11)) return false;   // the previous phase has been read
+            if (!MONA_IN_BOUNDS(stage_off + 128u <= EPI_BUF_BYTES, status, 104)) return false;
             #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 const uint32_t addr = epi_buf + stage_off + (((uint32_t)q ^ swz) << 4);
@@ -758,7 +766,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
                     #pragma unroll
                     for (int q = 0; q < 8; ++q) {
-                        if (row_ok && gc0 + 8 * q < p.N) cin_raw[q] = __ldcg(reinterpret_cast<const uint4*>(p.cin + row_off + gc0 + 8 * q));
+                        if (row_ok && gc0 + 8 * q < p.N && MONA_IN_BOUNDS(row_off + gc0 + 8 * q + 8 <= (long long)g.C * p.mat_stride, status, 105)) cin_raw[q] = __ldcg(reinterpret_cast<const uint4*>(p.cin + row_off + gc0 + 8 * q));
                         else cin_raw[q] = make_uint4(0u, 0u, 0u, 0u);
                     }
                 };
