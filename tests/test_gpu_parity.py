@@ -148,6 +148,22 @@ def test_ns_step_counts(T):
     check(errs, TOL_O_BF16)
 
 
+def test_more_iterations_than_one_launch_holds():
+    """T = 7: the Newton-Schulz kernel takes five iterations per launch, so this is two launches per chunk (5 + 2),
+    the second continuing on the first one's iterate."""
+    hp = pkg.default_hparams(ns_steps=7)
+    errs = run_case([(2, 256, 384), (1, 384, 256)], steps=2, hp=hp, seed=8)
+    check(errs, TOL_O_BF16)
+    assert errs["launches"] == 2 * 4        # per chunk: prologue, two Newton-Schulz launches, update
+
+
+def test_many_small_matrices_span_several_chunks():
+    """600 stacked 64x128 matrices: more than one chunk holds (512), one tile per GEMM and matrix, so the kernel's work
+    order and its per-matrix completion counters carry the whole load; a sample is followed by the oracle."""
+    errs = run_case([(600, 64, 128)], steps=2, seed=12, sample={0: [0, 1, 255, 511, 512, 599]})
+    check(errs, TOL_O_BF16)
+
+
 def test_fixed_scale_and_other_hyperparameters():
     hp = pkg.default_hparams(scale_mode=1, scale_value=0.37, lr=5e-3, momentum=0.8, weight_decay=0.0,
                              accel_beta=0.9, accel_alpha=-5.0)
