@@ -52,11 +52,11 @@ constexpr int TC_THREADS = 32 * EPI_WARP0 + TC_EPI_THREADS;       // 384
 // with the ~1.5 KiB of shared memory the kernel leaves, lets one 128-thread block of the elementwise kernels of the
 // NEXT chunk run beside it, so prologue and update overlap the GEMMs instead of waiting for the SMs).  Then the
 // warpgroup of the producer, MMA issuer, scheduler and store warp gives registers back and the two epilogue warpgroups
-// take them (setmaxnreg): 128 x 40 + 256 x 208 = 58368.  An epilogue thread can then hold its share of BOTH
+// take them (setmaxnreg): 128 x 56 + 256 x 200 = 58368.  An epilogue thread can then hold its share of BOTH
 // accumulators of a macro-tile.
 constexpr int TC_MAX_REGS = 152;
-constexpr int REGS_CONTROL = 40;
-constexpr int REGS_EPILOGUE = 208;
+constexpr int REGS_CONTROL = 56;
+constexpr int REGS_EPILOGUE = 200;
 constexpr int CTA_M = TC_BM / 2;                                  // accumulator rows held by one CTA
 constexpr int CTA_N = TC_BN / 2;                                  // B-operand rows one CTA stages per 256-column tile
 constexpr uint32_t BOX_BYTES = TC_BOX * TC_BOX * 2;               // 8 KiB
@@ -404,6 +404,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     // producer's view of the slab ring: next entry, next slab, oldest entry not yet known to be free, free slabs, and
     // the slabs every entry in flight took (3 bits each, wrap-around gap included)
     uint32_t ent = 0, slab_head = 0, tail_ent = 0, slabs_free = NSLAB;
+    uint32_t ent_e = 0, ent_par = 0, tail_e = 0, tail_par = 0;     // entries modulo NENT and their use parities, kept incrementally
     unsigned long long ent_cost = 0ull;
     const uint32_t full_leader = map_to_cta(bar_full, 0);
     auto produce = [&](const Item& it) -> bool {
@@ -430,17 +431,18 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             const uint32_t gap = slab_head + nslab > NSLAB ? NSLAB - slab_head : 0u;     // slabs skipped at the end of the ring
             const uint32_t need = gap + nslab;
             while (slabs_free < need) {        // entries are released in order: take back the oldest one's slabs
-                const uint32_t e = tail_ent % NENT;
-                if (!mbar_wait(bar_empty + 8 * e, (tail_ent / NENT) & 1u, abort_flag, status, 1)) return false;
-                slabs_free += (uint32_t)(ent_cost >> (3 * e)) & 7u;
+                if (!mbar_wait(bar_empty + 8 * tail_e, tail_par, abort_flag, status, 1)) return false;
+                slabs_free += (uint32_t)(ent_cost >> (3 * tail_e)) & 7u;
                 ++tail_ent;
+                if (++tail_e == NENT) { tail_e = 0; tail_par ^= 1u; }
             }
             slabs_free -= need;
-            const uint32_t e = ent % NENT;
+            const uint32_t e = ent_e;
             ent_cost = (ent_cost & ~(7ull << (3 * e))) | ((unsigned long long)need << (3 * e));
             const uint32_t pos = gap ? 0u : slab_head;
             slab_head = pos + nslab == NSLAB ? 0u : pos + nslab;
             ++ent;
+            if (++ent_e == NENT) { ent_e = 0; ent_par ^= 1u; }
             if (!MONA_IN_BOUNDS(pos + nslab <= NSLAB && e < NENT && it.c < g.C, status, 102)) return false;
             const uint32_t full = full_leader + 8 * e;
             const uint32_t sa = base + pos * SLAB_BYTES;
@@ -487,13 +489,15 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 ok = produce(it);
             }
             // stay until the tensor cores have released every k-slice: the commits arrive on this CTA's barriers
-            for (; ok && tail_ent < ent; ++tail_ent)
-                ok = mbar_wait(bar_empty + 8 * (tail_ent % NENT), (tail_ent / NENT) & 1u, abort_flag, status, 5);
+            for (; ok && tail_ent < ent; ++tail_ent) {
+                ok = mbar_wait(bar_empty + 8 * tail_e, tail_par, abort_flag, status, 5);
+                if (++tail_e == NENT) { tail_e = 0; tail_par ^= 1u; }
+            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
-            uint32_t ment = 0, mslab = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
+            uint32_t ment_e = 0, ment_par = 0, mslab = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
@@ -523,12 +527,12 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     // same slab walk as the producer's
                     const uint32_t pos = mslab + nslab > NSLAB ? 0u : mslab;
                     mslab = pos + nslab == NSLAB ? 0u : pos + nslab;
-                    const uint32_t e = ment % NENT;
+                    const uint32_t e = ment_e;
                     if (!MONA_IN_BOUNDS(pos + nslab <= NSLAB && tc.tm < p.tiles_m && tc.tn + tc.nsub <= p.tiles_n, status, 103)) { ok = false; break; }
                     const uint32_t stage_lo = (base + pos * SLAB_BYTES) >> 4;
                     // no tcgen05 fence here: the operands arrive through the asynchronous proxy and the barrier orders them
-                    if (!(ok = mbar_wait(bar_full + 8 * e, (ment / NENT) & 1u, abort_flag, status, 3))) break;
-                    ++ment;
+                    if (!(ok = mbar_wait(bar_full + 8 * e, ment_par, abort_flag, status, 3))) break;
+                    if (++ment_e == NENT) { ment_e = 0; ment_par ^= 1u; }
                     const uint32_t a_mn = kb >= a_switch ? 1u : 0u, b_mn0 = kb >= b_switch[0] ? 1u : 0u;
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
                     const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step0 = b_mn0 ? (2048u >> 4) : (32u >> 4);
