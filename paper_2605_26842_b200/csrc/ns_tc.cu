@@ -117,6 +117,14 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Hand-back of a ring slot whose 16 bytes this thread has loaded into `c, q, t, stop`: nothing is published, so the arrival
+// needs no release (at cluster scope that is a fence which waits for everything the thread has in flight - for the MMA issuer
+// its queued tensor-core work, a couple of thousand cycles per item); it must only not be issued before the load has returned.
+// The loaded words are never negative; folding their sign bit into the address makes the instruction depend on the load.
+__device__ __forceinline__ void mbar_arrive_slot_read(uint32_t cluster_addr, uint32_t c, uint32_t q, uint32_t t, uint32_t stop) {
+    const uint32_t zero = ((c | q | t | stop) >> 31) << 3;
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr + zero) : "memory");
+}
 // The same with the default semantics, for hand-overs that carry no shared-memory data (tensor-memory accumulators).
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -396,7 +404,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         const uint32_t slot = n % RING, par = (n / RING) & 1u;
         if (!mbar_wait<true>(bar_ring_full + 8 * slot, par, abort_flag, status, site)) return false;
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(it.c), "=r"(it.q), "=r"(it.t), "=r"(it.stop) : "r"(ring_items + 16 * slot) : "memory");
-        if (arrive) mbar_arrive_cluster(ring_empty_leader + 8 * slot);
+        if (arrive) mbar_arrive_slot_read(ring_empty_leader + 8 * slot, it.c, it.q, it.t, it.stop);
         return true;
     };
 
@@ -708,7 +716,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             Item it;
             if (!take_item(n, it, 10, false)) break;
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(ring_empty_leader + 8 * (n % RING));   // every lane has its copy of the item
+            if (lane == 0) mbar_arrive_slot_read(ring_empty_leader + 8 * (n % RING), it.c, it.q, it.t, it.stop);   // every lane has its copy of the item
             if (it.stop) break;
             const NsPhase& p = g.ph[it.q];
             const TileCoord tc = decode_tile(p, it.t);
