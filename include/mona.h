@@ -51,7 +51,8 @@ typedef enum {
     MONA_ERR_NONFINITE = 6,          /* ||M_k||_F of some matrix was inf/nan                          */
     MONA_ERR_ARCH = 7,               /* device is not compute capability 10.x                         */
     MONA_ERR_BUFFER_TOO_SMALL = 8,   /* state or workspace smaller than mona_query_sizes() reports    */
-    MONA_ERR_BOUNDS = 9              /* debug build (-DMONA_DEBUG) only: a kernel's index check failed */
+    MONA_ERR_BOUNDS = 9,             /* debug build (-DMONA_DEBUG) only: a kernel's index check failed */
+    MONA_ERR_NOT_BUILT = 10          /* the call needs a build option this library was compiled without */
 } mona_status;
 
 typedef enum { MONA_F32 = 0, MONA_BF16 = 1 } mona_dtype;
@@ -239,6 +240,42 @@ mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* d
 /* The work the iteration itself needs when both symmetric products are computed once per pair of entries:
  * 3 s^2 l + s^3 per matrix and iteration (tensor-core path only). */
 mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful);
+
+/* Profiling build only (library compiled with -DMONA_TRACE; every other build returns MONA_ERR_NOT_BUILT and
+ * touches nothing).  The paper has no counterpart: this is the instrument behind the per-role wait times quoted
+ * for the Newton-Schulz kernel.  In that build every role of the kernel (TMA producer, MMA issuer, scheduler,
+ * epilogue warps, store warp) adds up the SM clock cycles its waits took, and the MMA issuer the cycles and
+ * k-slices (64 of the inner dimension) per kind of tile; the arithmetic is unchanged, the kernel a few per
+ * cent slower.  One row of MONA_TRACE_SLOTS 64-bit words per CTA (row = block index; even rows are the CTAs
+ * that issue the MMAs and schedule), summed over all launches since the last reset.
+ * mona_trace_read() synchronises the device, copies the first `rows` rows (at most MONA_TRACE_ROWS) to the
+ * HOST array `out` (rows * MONA_TRACE_SLOTS words; may be NULL with rows = 0) and clears the table when
+ * `reset` is non-zero.  Not thread-safe against running steps of other threads. */
+#define MONA_TRACE_ROWS 160
+#define MONA_TRACE_SLOTS 64
+typedef enum mona_trace_slot {
+    MONA_TRACE_KERNEL = 0,            /* launch start to the end of the producer's role                        */
+    MONA_TRACE_PRODUCER_EMPTY = 1,    /* producer: waiting for free operand slabs                              */
+    MONA_TRACE_PRODUCER_RING = 2,     /* producer: waiting for the next published work item                    */
+    MONA_TRACE_PRODUCER_ROLE = 3,     /* producer: whole role                                                  */
+    MONA_TRACE_MMA_RING = 4,          /* MMA issuer: waiting for the next published work item                  */
+    MONA_TRACE_MMA_ROLE = 5,          /* MMA issuer: whole role                                                */
+    MONA_TRACE_SCHED_DEPENDENCY = 6,  /* scheduler: waiting for the previous GEMM of an item's matrix          */
+    MONA_TRACE_SCHED_SLOT = 7,        /* scheduler: waiting for a free slot of the item ring (it is ahead)     */
+    MONA_TRACE_SCHED_ROLE = 8,        /* scheduler: whole role                                                 */
+    MONA_TRACE_EPI_ACC_FULL = 9,      /* epilogue: waiting for a finished accumulator (sum over 8 warps)       */
+    MONA_TRACE_EPI_STAGE_EMPTY = 10,  /* epilogue: waiting for the staging buffer (sum over 8 warps)           */
+    MONA_TRACE_EPI_RING = 11,         /* epilogue: waiting for the next published item (sum over 8 warps)      */
+    MONA_TRACE_EPI_ROLE = 12,         /* epilogue: whole role (sum over 8 warps)                               */
+    MONA_TRACE_STORE_STAGED = 13,     /* store warp: waiting for a staged 128-column phase                     */
+    MONA_TRACE_STORE_ROLE = 14,       /* store warp: whole role                                                */
+    MONA_TRACE_ITEMS = 15,            /* work items completed by this CTA (a count, not cycles)                */
+    MONA_TRACE_TILE0 = 16             /* + 4 * kind + {0: cycles of the MMA issuer inside tiles of the kind, 1: their
+                                         k-slices (a count), 2: of the cycles, waiting for operands, 3: waiting for an
+                                         accumulator}; kind 0 / 1: X X^T off / on the diagonal, 2 / 3: b A + c A^2 + a I
+                                         off / on the diagonal, 4: 256 x 512 macro-tile of X' = B' X, 5: single tile of it */
+} mona_trace_slot;
+mona_status mona_trace_read(unsigned long long* out, size_t rows, int reset);
 
 /* Allocation-free prologue for ONE matrix.  The paper has no counterpart to this entry point; it exists
  * for integration reasons only.  It performs lines 4-7 and 10 of Algorithm 1 on a rows x cols matrix

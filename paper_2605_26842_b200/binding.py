@@ -13,7 +13,8 @@ _LIB_PATH = os.environ.get("MONA_LIBRARY") or os.path.join(_HERE, "libmona.so")
 
 STATUS_NAMES = {0: "MONA_OK", 1: "MONA_ERR_INVALID_ARG", 2: "MONA_ERR_UNSUPPORTED_SHAPE", 3: "MONA_ERR_ALIGNMENT",
                 4: "MONA_ERR_CUDA", 5: "MONA_ERR_TIMEOUT", 6: "MONA_ERR_NONFINITE", 7: "MONA_ERR_ARCH",
-                8: "MONA_ERR_BUFFER_TOO_SMALL", 9: "MONA_ERR_BOUNDS"}
+                8: "MONA_ERR_BUFFER_TOO_SMALL", 9: "MONA_ERR_BOUNDS", 10: "MONA_ERR_NOT_BUILT"}
+TRACE_ROWS, TRACE_SLOTS = 160, 64       # MONA_TRACE_ROWS, MONA_TRACE_SLOTS
 MONA_F32, MONA_BF16 = 0, 1
 MONA_STATE_COMBINED = 2      # single auxiliary buffer Z = beta_a A - (1 - beta_a) G
 
@@ -63,6 +64,7 @@ def lib() -> C.CDLL:
     L.mona_query_sizes_opt.argtypes = [C.POINTER(MatrixDesc), C.c_int64, C.POINTER(Options), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.mona_create_opt.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, C.POINTER(Options), vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_last_ns_useful_flops.argtypes = [vp, C.POINTER(C.c_double)]
+    L.mona_trace_read.argtypes = [C.POINTER(C.c_ulonglong), C.c_size_t, C.c_int]
     L.mona_create.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_step.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vp]
     L.mona_step_ex.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, C.c_uint32, vp]
@@ -80,10 +82,20 @@ def lib() -> C.CDLL:
     L.mona_destroy.restype = None
     for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_set_chunk_overlap", "mona_query_sizes", "mona_create", "mona_step",
                  "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops",
-                 "mona_default_options", "mona_query_sizes_opt", "mona_create_opt", "mona_last_ns_useful_flops"):
+                 "mona_default_options", "mona_query_sizes_opt", "mona_create_opt", "mona_last_ns_useful_flops", "mona_trace_read"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
+
+
+def trace_read(reset: bool = True, rows: int = TRACE_ROWS):
+    """mona_trace_read(): the profiling build's table as a list of `rows` lists of TRACE_SLOTS integers (row = CTA).
+    Raises MonaError(MONA_ERR_NOT_BUILT) unless the loaded library was compiled with -DMONA_TRACE."""
+    buf = (C.c_ulonglong * (rows * TRACE_SLOTS))()
+    st = lib().mona_trace_read(buf, rows, 1 if reset else 0)
+    if st:
+        raise MonaError(st, "mona_trace_read")
+    return [list(buf[r * TRACE_SLOTS:(r + 1) * TRACE_SLOTS]) for r in range(rows)]
 
 
 def default_hparams(**overrides) -> Hparams:

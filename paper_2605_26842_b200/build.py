@@ -10,6 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmona.so")
 LIB_DEBUG = os.path.join(HERE, "libmona_debug.so")      # -DMONA_DEBUG: kernels check their own indices
+LIB_TRACE = os.path.join(HERE, "libmona_trace.so")      # -DMONA_TRACE: the Newton-Schulz kernel accounts for its waits
 SOURCES = ["mona_api.cu", "elementwise.cu", "ns_fp32.cu", "ns_tc.cu"]
 
 
@@ -28,12 +29,15 @@ def needs_build(lib: str = LIB) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
-    lib = LIB_DEBUG if debug else LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False, trace: bool = False) -> str:
+    if debug and trace:
+        raise ValueError("one build variant at a time")
+    lib = LIB_DEBUG if debug else LIB_TRACE if trace else LIB
     if not force and not needs_build(lib):
         return lib
+    defines = ["-DMONA_DEBUG"] if debug else ["-DMONA_TRACE"] if trace else []
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-o", lib] + (["-DMONA_DEBUG"] if debug else []) + [os.path.join(CSRC, s) for s in SOURCES]
+           "-Xcompiler", "-fPIC", "-shared", "-o", lib] + defines + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -46,4 +50,4 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv, trace="--trace" in sys.argv))

@@ -719,6 +719,19 @@ mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful) {
     return MONA_OK;
 }
 
+static_assert(MONA_TRACE_ROWS == mona::NS_TRACE_ROWS && MONA_TRACE_SLOTS == mona::NS_TRACE_SLOTS &&
+              (int)MONA_TRACE_TILE0 == (int)mona::NS_TRACE_TILE0 && (int)MONA_TRACE_ITEMS == (int)mona::NS_TRACE_ITEMS &&
+              (int)MONA_TRACE_EPI_ROLE == (int)mona::NS_TRACE_EPI_ROLE && (int)MONA_TRACE_SCHED_ROLE == (int)mona::NS_TRACE_SCHED_ROLE,
+              "the public description of the profiling table follows the kernel's");
+
+mona_status mona_trace_read(unsigned long long* out, size_t rows, int reset) {
+    if (rows && !out) return MONA_ERR_INVALID_ARG;
+    int available = 0;
+    const cudaError_t e = mona::ns_trace_read(out, rows, reset, &available);
+    if (!available) return MONA_ERR_NOT_BUILT;
+    return e == cudaSuccess ? MONA_OK : MONA_ERR_CUDA;
+}
+
 const char* mona_last_error(const mona_handle* h) { return h ? h->last_error.c_str() : "null handle"; }
 
 void mona_destroy(mona_handle* h) {

@@ -85,6 +85,25 @@ static_assert(8 * (2 * NENT + 4 + 2 * RING + 2) + 16 + 16 * RING + 4 * NS_MAX_PH
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// ---- profiling build (-DMONA_TRACE) ---------------------------------------------------------------
+// Every role adds up, in registers, the cycles its waits took and flushes them once per work item into a per-CTA table
+// in shared memory; the MMA issuer also counts cycles and k-slices per kind of tile.  The tables are summed into
+// g_trace[blockIdx.x] when a launch ends and read back with ns_trace_read().  The arithmetic of the kernel is unchanged;
+// the clock reads cost a few per cent of its speed.  Without the flag all of this compiles to nothing.
+#ifdef MONA_TRACE
+__device__ unsigned long long g_trace[NS_TRACE_ROWS][NS_TRACE_SLOTS];
+__device__ __forceinline__ uint32_t trace_clock() {
+    uint32_t c;
+    asm volatile("mov.u32 %0, %%clock;" : "=r"(c));
+    return c;
+}
+#define TRACE_ONLY(...) __VA_ARGS__
+#define TRACE_PTR(x) (&(x))
+#else
+#define TRACE_ONLY(...)
+#define TRACE_PTR(x) nullptr
+#endif
+
 // ---- cluster --------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -159,14 +178,22 @@ __device__ __forceinline__ void latch_timeout(volatile int* abort_flag, DeviceSt
     status->timeout_site = site;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+// `waited` (profiling build only, may be null) accumulates the cycles spent here, the first attempt included.
 template <bool CLUSTER = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DeviceStatus* status,
-                                          unsigned site) {
-    if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
+                                          unsigned site, uint32_t* waited = nullptr) {
+    TRACE_ONLY(const uint32_t t_in = trace_clock();)
+    if (mbar_try_wait<CLUSTER>(bar, parity)) {
+        TRACE_ONLY(if (waited) *waited += trace_clock() - t_in;)
+        return true;
+    }
     const long long t0 = clock64();
     unsigned spins = 0;
     while (true) {
-        if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
+        if (mbar_try_wait<CLUSTER>(bar, parity)) {
+            TRACE_ONLY(if (waited) *waited += trace_clock() - t_in;)
+            return true;
+        }
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
@@ -183,12 +210,19 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned int* p) {
 }
 // Bounded wait until a dependency counter in global memory has reached `need` (acquire at device scope).
 __device__ __forceinline__ bool wait_counter(const unsigned int* ctr, unsigned need, volatile int* abort_flag,
-                                             DeviceStatus* status, unsigned site) {
-    if (ld_acquire_gpu(ctr) >= need) return true;
+                                             DeviceStatus* status, unsigned site, uint32_t* waited = nullptr) {
+    TRACE_ONLY(const uint32_t t_in = trace_clock();)
+    if (ld_acquire_gpu(ctr) >= need) {
+        TRACE_ONLY(if (waited) *waited += trace_clock() - t_in;)
+        return true;
+    }
     const long long t0 = clock64();
     unsigned spins = 0;
     while (true) {
-        if (ld_acquire_gpu(ctr) >= need) return true;
+        if (ld_acquire_gpu(ctr) >= need) {
+            TRACE_ONLY(if (waited) *waited += trace_clock() - t_in;)
+            return true;
+        }
         __nanosleep(64);
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
@@ -317,10 +351,6 @@ __device__ __forceinline__ TileCoord decode_tile(const NsPhase& p, int r) {
     return tc;
 }
 
-// A symmetric operand is stored as its lower block triangle: the k-slice [k0, k0 + 64) of row block
-// `blk` lies above the diagonal block exactly when it starts at or beyond the end of that block.
-__device__ __forceinline__ int fetch_transposed(int sym, int blk, int k0) { return sym && k0 >= (blk + 1) * TC_BM; }
-
 __device__ __forceinline__ uint4 pack8(const float* v) {
     uint4 r;
     __nv_bfloat162 t;
@@ -374,6 +404,12 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                    // 0: leader, 1: peer
     const int P = g.P;
+#ifdef MONA_TRACE
+    __shared__ unsigned long long s_trace[NS_TRACE_SLOTS];
+    const uint32_t t_kernel0 = trace_clock();
+    if (threadIdx.x < NS_TRACE_SLOTS) s_trace[threadIdx.x] = 0ull;
+    auto trace_add = [&](int slot, uint32_t v) { atomicAdd(&s_trace[slot], (unsigned long long)v); };
+#endif
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -400,9 +436,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
 
     // A reader's view of the item ring: wait for the n-th published item, copy it, hand the slot back.
     const uint32_t ring_empty_leader = map_to_cta(bar_ring_empty, 0);
-    auto take_item = [&](unsigned n, Item& it, unsigned site, bool arrive) -> bool {
+    auto take_item = [&](unsigned n, Item& it, unsigned site, bool arrive, uint32_t* waited = nullptr) -> bool {
         const uint32_t slot = n % RING, par = (n / RING) & 1u;
-        if (!mbar_wait<true>(bar_ring_full + 8 * slot, par, abort_flag, status, site)) return false;
+        if (!mbar_wait<true>(bar_ring_full + 8 * slot, par, abort_flag, status, site, waited)) return false;
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(it.c), "=r"(it.q), "=r"(it.t), "=r"(it.stop) : "r"(ring_items + 16 * slot) : "memory");
         if (arrive) mbar_arrive_slot_read(ring_empty_leader + 8 * slot, it.c, it.q, it.t, it.stop);
         return true;
@@ -414,6 +450,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     uint32_t ent = 0, slab_head = 0, tail_ent = 0, slabs_free = NSLAB;
     uint32_t ent_e = 0, ent_par = 0, tail_e = 0, tail_par = 0;     // entries modulo NENT and their use parities, kept incrementally
     unsigned long long ent_cost = 0ull;
+    TRACE_ONLY(uint32_t w_empty = 0;)
     const uint32_t full_leader = map_to_cta(bar_full, 0);
     auto produce = [&](const Item& it) -> bool {
         const NsPhase& p = g.ph[it.q];
@@ -439,7 +476,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             const uint32_t gap = slab_head + nslab > NSLAB ? NSLAB - slab_head : 0u;     // slabs skipped at the end of the ring
             const uint32_t need = gap + nslab;
             while (slabs_free < need) {        // entries are released in order: take back the oldest one's slabs
-                if (!mbar_wait(bar_empty + 8 * tail_e, tail_par, abort_flag, status, 1)) return false;
+                if (!mbar_wait(bar_empty + 8 * tail_e, tail_par, abort_flag, status, 1, TRACE_PTR(w_empty))) return false;
                 slabs_free += (uint32_t)(ent_cost >> (3 * tail_e)) & 7u;
                 ++tail_ent;
                 if (++tail_e == NENT) { tail_e = 0; tail_par ^= 1u; }
@@ -489,13 +526,16 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer (both CTAs) ----------------
+            TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_ring = 0;)
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
-                if (!(ok = take_item(n, it, 8, true)) || it.stop) break;
+                if (!(ok = take_item(n, it, 8, true, TRACE_PTR(w_ring))) || it.stop) break;
                 fence_proxy_async();       // the scheduler's acquire of the dependency precedes these copies
                 ok = produce(it);
+                TRACE_ONLY(trace_add(NS_TRACE_PRODUCER_EMPTY, w_empty); trace_add(NS_TRACE_PRODUCER_RING, w_ring); w_empty = w_ring = 0;)
             }
+            TRACE_ONLY(trace_add(NS_TRACE_PRODUCER_RING, w_ring); trace_add(NS_TRACE_PRODUCER_ROLE, trace_clock() - t_role0);)
             // stay until the tensor cores have released every k-slice: the commits arrive on this CTA's barriers
             for (; ok && tail_ent < ent; ++tail_ent) {
                 ok = mbar_wait(bar_empty + 8 * tail_e, tail_par, abort_flag, status, 5);
@@ -506,10 +546,12 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         // ---------------- MMA issuer (leader CTA only) ----------------
         if (lane == 0 && rank == 0) {
             uint32_t ment_e = 0, ment_par = 0, mslab = 0, acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
+            TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_ring = 0;)
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
-                if (!(ok = take_item(n, it, 9, true)) || it.stop) break;
+                if (!(ok = take_item(n, it, 9, true, TRACE_PTR(w_ring))) || it.stop) break;
+                TRACE_ONLY(const uint32_t t_item0 = trace_clock(); uint32_t w_full = 0, w_acc = 0;)
                 const NsPhase& p = g.ph[it.q];
                 const TileCoord tc = decode_tile(p, it.t);
                 const bool shared_ab = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
@@ -526,7 +568,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const uint32_t b_off0 = shared_ab ? 0u : (A_STAGE_BYTES >> 4);             // operand offsets inside a stage, in 16-byte units
                 const uint32_t b_off1 = (A_STAGE_BYTES + B_SUB_BYTES) >> 4;
                 // an accumulator must have been drained by the epilogue of its previous tile before the first MMA into it
-                if (!(ok = mbar_wait(bar_acc_empty + 8 * acc0, ((acc_par >> acc0) & 1u) ^ 1u, abort_flag, status, 2))) break;
+                if (!(ok = mbar_wait(bar_acc_empty + 8 * acc0, ((acc_par >> acc0) & 1u) ^ 1u, abort_flag, status, 2, TRACE_PTR(w_acc)))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + acc0 * TC_BN, d1 = d0 + TC_BN;
                 uint32_t accum = 0u;
@@ -539,7 +581,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     if (!MONA_IN_BOUNDS(pos + nslab <= NSLAB && tc.tm < p.tiles_m && tc.tn + tc.nsub <= p.tiles_n, status, 103)) { ok = false; break; }
                     const uint32_t stage_lo = (base + pos * SLAB_BYTES) >> 4;
                     // no tcgen05 fence here: the operands arrive through the asynchronous proxy and the barrier orders them
-                    if (!(ok = mbar_wait(bar_full + 8 * e, ment_par, abort_flag, status, 3))) break;
+                    if (!(ok = mbar_wait(bar_full + 8 * e, ment_par, abort_flag, status, 3, TRACE_PTR(w_full)))) break;
                     if (++ment_e == NENT) { ment_e = 0; ment_par ^= 1u; }
                     const uint32_t a_mn = kb >= a_switch ? 1u : 0u, b_mn0 = kb >= b_switch[0] ? 1u : 0u;
                     // one k-step of 16 advances 32 B inside the swizzle row (K-major) or 16 rows = 2048 B (MN-major)
@@ -554,7 +596,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                     if (tc.nsub == 2) {
                         if (kb == 0) {
-                            if (!(ok = mbar_wait(bar_acc_empty + 8 * (acc0 + 1), ((acc_par >> (acc0 + 1)) & 1u) ^ 1u, abort_flag, status, 2))) break;
+                            if (!(ok = mbar_wait(bar_acc_empty + 8 * (acc0 + 1), ((acc_par >> (acc0 + 1)) & 1u) ^ 1u, abort_flag, status, 2, TRACE_PTR(w_acc)))) break;
                             tc_fence_after();
                         }
                         const uint32_t b_mn1 = kb >= b_switch[1] ? 1u : 0u;
@@ -575,7 +617,17 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     acc_par ^= 1u << acc;
                 }
                 if (tc.nsub == 1) acc_next ^= 1u;
+#ifdef MONA_TRACE
+                {   // kind of tile: 0/1 X X^T off/on the diagonal, 2/3 b A + c A^2 + a I off/on the diagonal, 4 macro-tile, 5 single tile of X' = B' X
+                    const int kind = !p.symmetric ? (tc.nsub == 2 ? 4 : 5) : ((p.cin ? 2 : 0) + (shared_ab ? 1 : 0));
+                    const int slot = NS_TRACE_TILE0 + 4 * kind;
+                    trace_add(slot, trace_clock() - t_item0); trace_add(slot + 1, (uint32_t)num_kb);
+                    trace_add(slot + 2, w_full); trace_add(slot + 3, w_acc);
+                    trace_add(NS_TRACE_MMA_RING, w_ring); w_ring = 0;
+                }
+#endif
             }
+            TRACE_ONLY(trace_add(NS_TRACE_MMA_RING, w_ring); trace_add(NS_TRACE_MMA_ROLE, trace_clock() - t_role0);)
         }
     } else if (warp == STORE_WARP) {
         if (lane == 0) {
@@ -585,6 +637,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             // done for its matrix and phase once all of its stores have completed.  The epilogue warps never wait for global
             // memory.  It walks the items and their phases in the epilogue's order.
             uint32_t staged = 0;
+            TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_stg = 0;)
             bool ok = true;
             for (unsigned n = 0; ok; ++n) {
                 Item it;
@@ -599,7 +652,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                         const int x0 = (tc.tn + u) * TC_BN + ph * EPI_COLS;
                         if (x0 >= p.N) continue;
                         if (!MONA_IN_BOUNDS(m0 < p.M + CTA_M && it.c < g.C && tc.tm < p.tiles_m, status, 106)) { ok = false; break; }
-                        if (!(ok = mbar_wait(bar_stg_full, staged & 1u, abort_flag, status, 13))) break;
+                        if (!(ok = mbar_wait(bar_stg_full, staged & 1u, abort_flag, status, 13, TRACE_PTR(w_stg)))) break;
                         ++staged;
                         #pragma unroll
                         for (int bx = 0; bx < 2; ++bx) {
@@ -616,8 +669,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 fence_proxy_async();
                 __threadfence();
                 atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
+                TRACE_ONLY(trace_add(NS_TRACE_STORE_STAGED, w_stg); w_stg = 0; trace_add(NS_TRACE_ITEMS, 1u);)
             }
             bulk_wait_all();           // shared memory must outlive the stores that read it
+            TRACE_ONLY(trace_add(NS_TRACE_STORE_ROLE, trace_clock() - t_role0);)
         }
     } else if (warp == SCHED_WARP) {
         if (lane == 0 && rank == 0) {
@@ -653,11 +708,12 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 if (!it.stop && it.q > 0) { ctr = g.done + (size_t)it.c * P + (it.q - 1); need = 2u * phase_items[it.q - 1]; }
             };
             unsigned published = 0;
+            TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_slot = 0, w_dep = 0;)
             bool ok = true;
             while (ok) {
                 // an item is taken only once a ring slot is free for it: items stay in the common pool as long as possible
                 const uint32_t slot = published % RING, par = (published / RING) & 1u;
-                if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7))) break;
+                if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7, TRACE_PTR(w_slot)))) break;
                 const unsigned idx = atomicAdd(g.work_counter, 1u);
                 Item it;
                 decode(idx, it);
@@ -667,15 +723,17 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 }
                 const unsigned int* ctr; unsigned need;
                 dependency(it, ctr, need);
-                if (ctr && !(ok = wait_counter(ctr, need, abort_flag, status, 6))) break;
+                if (ctr && !(ok = wait_counter(ctr, need, abort_flag, status, 6, TRACE_PTR(w_dep)))) break;
                 fence_proxy_async();
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
                 asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
                 mbar_arrive_cluster(ring_full_own + 8 * slot);
                 mbar_arrive_cluster(ring_full_peer + 8 * slot);
                 ++published;
+                TRACE_ONLY(trace_add(NS_TRACE_SCHED_SLOT, w_slot); trace_add(NS_TRACE_SCHED_DEPENDENCY, w_dep); w_slot = w_dep = 0;)
                 if (it.stop) break;
             }
+            TRACE_ONLY(trace_add(NS_TRACE_SCHED_ROLE, trace_clock() - t_role0);)
         }
     }
     } else {
@@ -696,10 +754,11 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         const uint32_t swz = (uint32_t)row_in_cta & 7u;
         uint32_t acc_next = 0, acc_par = 0;   // acc_par: one use-parity bit per accumulator
         uint32_t staged = 0;                  // staging phases handed to the store warp so far
+        TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_ring = 0, w_accf = 0, w_stge = 0;)
         bool alive = true;
         // 128 packed columns of this thread's row go to the staging buffer; the store warp sends them on
         auto put_phase = [&](const uint4* pk) -> bool {
-            if (!mbar_wait(bar_stg_empty, (staged & 1u) ^ 1u, abort_flag, status, 11)) return false;   // the previous phase has been read
+            if (!mbar_wait(bar_stg_empty, (staged & 1u) ^ 1u, abort_flag, status, 11, TRACE_PTR(w_stge))) return false;   // the previous phase has been read
             if (!MONA_IN_BOUNDS(stage_off + 128u <= EPI_BUF_BYTES, status, 104)) return false;
             #pragma unroll
             for (int q = 0; q < 8; ++q) {
@@ -714,7 +773,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         };
         for (unsigned n = 0; alive; ++n) {
             Item it;
-            if (!take_item(n, it, 10, false)) break;
+            if (!take_item(n, it, 10, false, TRACE_PTR(w_ring))) break;
             __syncwarp();
             if (lane == 0) mbar_arrive_slot_read(ring_empty_leader + 8 * (n % RING), it.c, it.q, it.t, it.stop);   // every lane has its copy of the item
             if (it.stop) break;
@@ -739,7 +798,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     if (u < tc.nsub && alive) {
                         const uint32_t acc = acc0 + u;
                         const int n0 = (tc.tn + u) * TC_BN;
-                        if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { alive = false; break; }
+                        if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4, TRACE_PTR(w_accf))) { alive = false; break; }
                         tc_fence_after();
                         acc_par ^= 1u << acc;
                         const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
@@ -783,7 +842,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                 };
                 if (p.cin) load_cin(0);
-                if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4)) { alive = false; break; }
+                if (!mbar_wait(bar_acc_full + 8 * acc, (acc_par >> acc) & 1u, abort_flag, status, 4, TRACE_PTR(w_accf))) { alive = false; break; }
                 tc_fence_after();
                 acc_par ^= 1u << acc;
                 const uint32_t t_base = tmem_base + lane_base + acc * TC_BN + half * 64;
@@ -845,12 +904,21 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 }
             }
             if (tc.nsub == 1) acc_next ^= 1u;
+#ifdef MONA_TRACE
+            if (lane == 0) {      // one lane per warp: the table holds sums over the eight epilogue warps
+                trace_add(NS_TRACE_EPI_RING, w_ring); trace_add(NS_TRACE_EPI_ACC_FULL, w_accf); trace_add(NS_TRACE_EPI_STAGE_EMPTY, w_stge);
+            }
+            w_ring = w_accf = w_stge = 0;
+#endif
         }
+        TRACE_ONLY(if (lane == 0) trace_add(NS_TRACE_EPI_ROLE, trace_clock() - t_role0);)
     }
 
+    TRACE_ONLY(if (threadIdx.x == 0) trace_add(NS_TRACE_KERNEL, trace_clock() - t_kernel0);)
     if (*abort_flag) __nanosleep(200000);      // let copies that are still in flight land before the CTA goes away
     tc_fence_before();
     __syncthreads();
+    TRACE_ONLY(if (threadIdx.x < NS_TRACE_SLOTS) atomicAdd(&g_trace[blockIdx.x % NS_TRACE_ROWS][threadIdx.x], s_trace[threadIdx.x]);)
     cluster_sync();                            // neither CTA leaves (or frees tensor memory) while its peer may still signal it
     tc_fence_after();
     if (warp == 1) {
@@ -860,6 +928,25 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
 }
 
 }  // namespace
+
+cudaError_t ns_trace_read(unsigned long long* out, size_t rows, int reset, int* available) {
+#ifdef MONA_TRACE
+    *available = 1;
+    if (rows > (size_t)NS_TRACE_ROWS) rows = NS_TRACE_ROWS;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess && out && rows) e = cudaMemcpyFromSymbol(out, g_trace, rows * NS_TRACE_SLOTS * sizeof(unsigned long long));
+    if (e == cudaSuccess && reset) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_trace);
+        if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(unsigned long long) * NS_TRACE_ROWS * NS_TRACE_SLOTS);
+    }
+    return e;
+#else
+    (void)out; (void)rows; (void)reset;
+    *available = 0;
+    return cudaSuccess;
+#endif
+}
 
 void ns_phase_plan(NsPhase& p) {
     p.tiles_m = (p.M + TC_BM - 1) / TC_BM;

@@ -70,6 +70,33 @@ struct NsProgram {
                                 //    report STATUS_TIMEOUT and leave cleanly (all copies still complete; nothing faults)
 };
 
+// Layout of the profiling build's table (-DMONA_TRACE): one row per CTA (blockIdx.x; even rows are the leaders, which
+// alone run the MMA issuer and the scheduler), NS_TRACE_SLOTS 64-bit words per row, all in SM clock cycles unless noted,
+// summed over the launches since the last reset.
+constexpr int NS_TRACE_ROWS = 160;
+constexpr int NS_TRACE_SLOTS = 64;
+enum NsTraceSlot {
+    NS_TRACE_KERNEL = 0,            // launch start to the end of the producer's role
+    NS_TRACE_PRODUCER_EMPTY = 1,    // producer: waiting for free operand slabs
+    NS_TRACE_PRODUCER_RING = 2,     // producer: waiting for the next published item
+    NS_TRACE_PRODUCER_ROLE = 3,     // producer: whole role
+    NS_TRACE_MMA_RING = 4,          // MMA issuer: waiting for the next published item
+    NS_TRACE_MMA_ROLE = 5,          // MMA issuer: whole role
+    NS_TRACE_SCHED_DEPENDENCY = 6,  // scheduler: waiting for the previous phase of an item's matrix
+    NS_TRACE_SCHED_SLOT = 7,        // scheduler: waiting for a free slot of the item ring (it is ahead of the pipeline)
+    NS_TRACE_SCHED_ROLE = 8,        // scheduler: whole role
+    NS_TRACE_EPI_ACC_FULL = 9,      // epilogue: waiting for a finished accumulator (sum over the 8 warps)
+    NS_TRACE_EPI_STAGE_EMPTY = 10,  // epilogue: waiting for the staging buffer (sum over the 8 warps)
+    NS_TRACE_EPI_RING = 11,         // epilogue: waiting for the next published item (sum over the 8 warps)
+    NS_TRACE_EPI_ROLE = 12,         // epilogue: whole role (sum over the 8 warps)
+    NS_TRACE_STORE_STAGED = 13,     // store warp: waiting for a staged phase
+    NS_TRACE_STORE_ROLE = 14,       // store warp: whole role
+    NS_TRACE_ITEMS = 15,            // work items completed by this CTA (a count)
+    NS_TRACE_TILE0 = 16             // 6 kinds of tile x {cycles of the MMA issuer inside the tile, k-slices (a count), of which
+                                    // waiting for operands, of which waiting for an accumulator}; kinds: 0/1 X X^T off/on the
+                                    // diagonal, 2/3 b A + c A^2 + a I off/on the diagonal, 4 macro-tile and 5 single tile of X' = B' X
+};
+
 struct alignas(64) NsMaps {
     CUtensorMap m[NS_MAPS];
 };
@@ -94,6 +121,9 @@ inline size_t ns_sched_words(int C, int P) { return 64 + (size_t)C * P; }
 // Sets the kernel's shared-memory attribute and finds how many CTA pairs the device holds at once.
 // Call once per device before the first launch.
 cudaError_t ns_configure(int* max_pairs);
+// Copies the first `rows` rows of the profiling table to `out` (host) after synchronising the device, and clears the table
+// when `reset` is set.  *available = 0 (and nothing else happens) unless the library was built with -DMONA_TRACE.
+cudaError_t ns_trace_read(unsigned long long* out, size_t rows, int reset, int* available);
 cudaError_t launch_ns_program(const NsMaps& maps, const NsProgram& g, const NsUpdatePtrs& upd, int max_pairs,
                               DeviceStatus* status, cudaStream_t stream);
 
