@@ -131,7 +131,7 @@ mona_status mona_default_hparams(mona_hparams* hp);
  *                        benchmark sets: a thread owns a row of the accumulator, so its fp32 read-modify-write of W
  *                        touches 32 lines per warp instruction and sits, unhidden, in the macro-tile's epilogue.
  *   ns_delay           : how many matrices apart consecutive Newton-Schulz GEMMs of one matrix sit in the kernel's
- *                        work order (0 = the default, 6; at most 1024; a value >= the chunk's matrix count
+ *                        work order (0 = the default, 20; at most 1024; a value >= the chunk's matrix count
  *                        runs the chunk GEMM by GEMM).  Larger values hide the dependency latency
  *                        better, smaller ones keep intermediates closer to the cache.  Results do not depend on it.
  *   macro_tile_min_k   : X' = B' X runs as 256 x 512 macro-tiles (two tiles sharing one staged operand slice, both

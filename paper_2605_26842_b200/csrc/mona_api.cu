@@ -252,7 +252,7 @@ mona_status mona_default_options(mona_options* opt) {
     opt->chunk_budget_bytes = g_chunk_budget_bytes.load();
     opt->chunk_overlap = g_chunk_overlap.load();
     opt->fuse_update = 0;
-    opt->ns_delay = 6;
+    opt->ns_delay = 20;
     opt->macro_tile_min_k = 1;
     return MONA_OK;
 }

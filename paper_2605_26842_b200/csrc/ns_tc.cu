@@ -81,7 +81,7 @@ constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
 // epilogue warps in the peer
 constexpr uint32_t RING_READERS = 3 + TC_EPI_WARPS + 2 + TC_EPI_WARPS;
 static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-static_assert(8 * (2 * NENT + 4 + 2 * RING + 2) + 16 + 16 * RING + 4 * NS_MAX_PHASES <= SMEM_CTRL_BYTES, "control block");
+static_assert(8 * (2 * NENT + 4 + 2 * RING + 2) + 16 + 16 * RING + 4 * (NS_MAX_PHASES + 1) <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -129,9 +129,11 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
-// Arrive (release at cluster scope) on a barrier given by its cluster-wide address (own CTA or the peer).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+// Publication of shared-memory data to both CTAs of the pair: ONE release fence at cluster scope, then an arrival without
+// semantics of its own per barrier (a release on each arrival would be a second fence of the same cost).
+__device__ __forceinline__ void fence_release_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive_relaxed_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -255,7 +257,10 @@ __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Orders this thread's earlier generic-proxy accesses (plain loads/stores, acquire loads) with later accesses
 // through the asynchronous proxy (TMA), and the other way round.
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// Orders this thread's accesses through the generic proxy against its accesses through the asynchronous proxy (TMA), for
+// one state space only: the unqualified fence costs over a thousand cycles wherever it stands.
+__device__ __forceinline__ void fence_proxy_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (64 bits) for a 128-byte-swizzled bf16 tile whose rows are 128 bytes long and
 // stacked densely (what a 64-wide TMA box with SWIZZLE_128B produces):
@@ -396,7 +401,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const uint32_t bar_stg_empty = bar_stg_full + 8;            // staging buffer read by the stores (store warp)
     const uint32_t tmem_slot = bar_stg_empty + 8;               // 4 B + abort flag 4 B + 8 B pad
     const uint32_t ring_items = tmem_slot + 16;                 // RING x 16 B
-    volatile unsigned int* phase_items = reinterpret_cast<volatile unsigned int*>(smem_raw + (ring_items + 16 * RING - smem_u32(smem_raw)));   // NS_MAX_PHASES x 4 B
+    // items per matrix of the phases before phase q (q = 0 .. P): phase q has phase_first[q + 1] - phase_first[q] items
+    volatile unsigned int* phase_first = reinterpret_cast<volatile unsigned int*>(smem_raw + (ring_items + 16 * RING - smem_u32(smem_raw)));   // (NS_MAX_PHASES + 1) x 4 B
     uint8_t* ctrl_ptr = smem_raw + (ctrl - smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(ctrl_ptr + (tmem_slot - ctrl));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl_ptr + (tmem_slot - ctrl) + 4);
@@ -413,7 +419,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int q = 0; q < NS_MAX_PHASES; ++q) phase_items[q] = q < P ? (unsigned)g.ph[q].items_per_mat : 0u;
+        unsigned first = 0u;
+        for (int q = 0; q <= NS_MAX_PHASES; ++q) { phase_first[q] = first; if (q < P) first += (unsigned)g.ph[q].items_per_mat; }
         for (int s = 0; s < NENT; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
@@ -531,7 +538,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             for (unsigned n = 0; ok; ++n) {
                 Item it;
                 if (!(ok = take_item(n, it, 8, true, TRACE_PTR(w_ring))) || it.stop) break;
-                fence_proxy_async();       // the scheduler's acquire of the dependency precedes these copies
+                fence_proxy_async_global();       // the scheduler's acquire of the dependency precedes these copies
                 ok = produce(it);
                 TRACE_ONLY(trace_add(NS_TRACE_PRODUCER_EMPTY, w_empty); trace_add(NS_TRACE_PRODUCER_RING, w_ring); w_empty = w_ring = 0;)
             }
@@ -666,7 +673,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 }
                 if (!ok) break;
                 bulk_wait_all();                           // the item's output is in global memory
-                fence_proxy_async();
+                fence_proxy_async_global();
                 __threadfence();
                 atomicAdd(g.done + (size_t)it.c * P + it.q, 1u);
                 TRACE_ONLY(trace_add(NS_TRACE_STORE_STAGED, w_stg); w_stg = 0; trace_add(NS_TRACE_ITEMS, 1u);)
@@ -680,55 +687,68 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             const uint32_t ring_items_peer = map_to_cta(ring_items, 1), ring_full_peer = map_to_cta(bar_ring_full, 1);
             const uint32_t ring_full_own = map_to_cta(bar_ring_full, 0);
             // Item order: for tau = 0, 1, ...: for q = 0 .. P-1: the items of phase q of matrix c = tau - delay * q, where that
-            // matrix exists.  The cursor (tau, q, index of the group's first item) only moves forward; per-phase item counts
-            // come from shared memory, and the q range that has a matrix at this tau is computed, not searched.
-            int cur_tau = 0, cur_q = 0;
+            // matrix exists, i.e. for q_lo(tau) <= q <= q_hi(tau) with q_hi = min(P - 1, tau / delay) (c >= 0) and
+            // q_lo = ceil((tau - C + 1) / delay) (c < C).  The cursor (tau, index of the first item of its group of phases)
+            // only moves forward, a whole tau at a time; q_lo and q_hi are kept incrementally, so that finding an item costs
+            // a few shared-memory reads however many items the other pairs have taken since this pair's last one.
+            const int C = g.C, delay = g.delay;
+            int cur_tau = 0, q_lo = 0, q_hi = 0, lo_cnt = 0, hi_cnt = 0;
             unsigned cur_base = 0;
-            auto decode = [&](unsigned idx, Item& it) {
+            auto decode = [&](unsigned idx, Item& it) -> bool {
                 it.stop = idx >= g.total_items ? 1 : 0;
                 it.c = it.q = it.t = 0;
-                if (it.stop) return;
+                if (it.stop) return true;
                 while (true) {
-                    const int over = cur_tau - g.C + 1;                                 // c < C  <=>  q >= over / delay (rounded up)
-                    const int q_lo = over > 0 ? (over + g.delay - 1) / g.delay : 0;
-                    int q_hi = cur_tau / g.delay;                                        // c >= 0
-                    if (q_hi > P - 1) q_hi = P - 1;
-                    if (cur_q < q_lo) cur_q = q_lo;
-                    if (cur_q > q_hi) { ++cur_tau; cur_q = 0; continue; }
-                    const unsigned n = phase_items[cur_q];
-                    if (idx < cur_base + n) { it.c = cur_tau - g.delay * cur_q; it.q = cur_q; it.t = (int)(idx - cur_base); return; }
-                    cur_base += n;
-                    ++cur_q;
+                    const unsigned n_tau = q_lo <= q_hi ? phase_first[q_hi + 1] - phase_first[q_lo] : 0u;
+                    if (idx < cur_base + n_tau) break;
+                    if (cur_tau >= C + P * delay) return false;          // past the last group: the item count and this walk disagree
+                    cur_base += n_tau;
+                    ++cur_tau;
+                    if (++hi_cnt == delay) { hi_cnt = 0; if (q_hi < P - 1) ++q_hi; }
+                    if (cur_tau == C) { q_lo = 1; lo_cnt = 0; }
+                    else if (cur_tau > C && ++lo_cnt == delay) { lo_cnt = 0; ++q_lo; }
                 }
+                const unsigned r = idx - cur_base + phase_first[q_lo];      // counted from phase 0 of this tau
+                int q = q_lo;
+                while (phase_first[q + 1] <= r) ++q;                        // ends at q <= q_hi since r < phase_first[q_hi + 1]
+                it.q = q;
+                it.t = (int)(r - phase_first[q]);
+                it.c = cur_tau - delay * q;
+                return true;
             };
             // The phase before an item must be complete for its matrix: its outputs are the item's operands, and the buffers
             // the item overwrites were last read two phases further back.
             auto dependency = [&](const Item& it, const unsigned int*& ctr, unsigned& need) {
                 ctr = nullptr; need = 0u;
-                if (!it.stop && it.q > 0) { ctr = g.done + (size_t)it.c * P + (it.q - 1); need = 2u * phase_items[it.q - 1]; }
+                if (!it.stop && it.q > 0) { ctr = g.done + (size_t)it.c * P + (it.q - 1); need = 2u * (phase_first[it.q] - phase_first[it.q - 1]); }
             };
             unsigned published = 0;
             TRACE_ONLY(const uint32_t t_role0 = trace_clock(); uint32_t w_slot = 0, w_dep = 0;)
             bool ok = true;
+            // The counter is always asked for one item more than has been published, so that its round trip (as long as that
+            // of the dependency check) runs beside the dependency wait of the item before.  An item claimed early is still
+            // published in order and only after everything it depends on, all of it with smaller indices, is complete.
+            unsigned next_idx = atomicAdd(g.work_counter, 1u);
             while (ok) {
-                // an item is taken only once a ring slot is free for it: items stay in the common pool as long as possible
                 const uint32_t slot = published % RING, par = (published / RING) & 1u;
                 if (!(ok = mbar_wait<true>(bar_ring_empty + 8 * slot, par ^ 1u, abort_flag, status, 7, TRACE_PTR(w_slot)))) break;
-                const unsigned idx = atomicAdd(g.work_counter, 1u);
+                const unsigned idx = next_idx;
+                if (idx < g.total_items) next_idx = atomicAdd(g.work_counter, 1u);
                 Item it;
-                decode(idx, it);
-                if (!it.stop && !MONA_IN_BOUNDS(it.c >= 0 && it.c < g.C && it.q >= 0 && it.q < P && it.t >= 0 && (unsigned)it.t < phase_items[it.q], status, 101)) {
+                const bool found = decode(idx, it);
+                if (!found || !it.stop && !MONA_IN_BOUNDS(it.c >= 0 && it.c < g.C && it.q >= 0 && it.q < P && it.t >= 0 && (unsigned)it.t < phase_first[it.q + 1] - phase_first[it.q], status, 101)) {
                     latch_timeout(abort_flag, status, 101);        // an item that does not exist: give up the launch, cleanly
                     break;
                 }
                 const unsigned int* ctr; unsigned need;
                 dependency(it, ctr, need);
                 if (ctr && !(ok = wait_counter(ctr, need, abort_flag, status, 6, TRACE_PTR(w_dep)))) break;
-                fence_proxy_async();
+                // (no proxy fence here: this thread issues no copy; the producers fence after they have taken the item)
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
                 asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ring_items_peer + 16 * slot), "r"(it.c), "r"(it.q), "r"(it.t), "r"(it.stop) : "memory");
-                mbar_arrive_cluster(ring_full_own + 8 * slot);
-                mbar_arrive_cluster(ring_full_peer + 8 * slot);
+                fence_release_cluster();       // the item, and the acquire of its dependency before it, precede both arrivals
+                mbar_arrive_relaxed_cluster(ring_full_own + 8 * slot);
+                mbar_arrive_relaxed_cluster(ring_full_peer + 8 * slot);
                 ++published;
                 TRACE_ONLY(trace_add(NS_TRACE_SCHED_SLOT, w_slot); trace_add(NS_TRACE_SCHED_DEPENDENCY, w_dep); w_slot = w_dep = 0;)
                 if (it.stop) break;
@@ -765,7 +785,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const uint32_t addr = epi_buf + stage_off + (((uint32_t)q ^ swz) << 4);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pk[q].x), "r"(pk[q].y), "r"(pk[q].z), "r"(pk[q].w) : "memory");
             }
-            fence_proxy_async();                   // generic-proxy writes above must be visible to the TMA engine
+            fence_proxy_async_shared();            // generic-proxy writes above must be visible to the TMA engine
             __syncwarp();
             if (lane == 0) mbar_arrive_local(bar_stg_full);
             ++staged;
