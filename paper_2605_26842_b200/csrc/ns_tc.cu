@@ -81,7 +81,7 @@ constexpr long long WAIT_BUDGET_CYCLES = 1000000000ll;            // ~0.5 s
 // epilogue warps in the peer
 constexpr uint32_t RING_READERS = 3 + TC_EPI_WARPS + 2 + TC_EPI_WARPS;
 static_assert(SMEM_TOTAL <= 232448, "shared memory budget");
-static_assert(8 * (2 * NENT + 4 + 2 * RING + 2) + 16 + 16 * RING + 4 * (NS_MAX_PHASES + 1) <= SMEM_CTRL_BYTES, "control block");
+static_assert(8 * (2 * NENT + 4 + 2 * RING + 4) + 16 + 16 * RING + 4 * (NS_MAX_PHASES + 1) <= SMEM_CTRL_BYTES, "control block");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -252,11 +252,11 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all earlier store groups of this thread have finished READING shared memory (the staging buffer may be rewritten)
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// (all but the PENDING most recent groups)
+template <int PENDING>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(PENDING) : "memory"); }
 // all earlier store groups of this thread have completed (their global writes are done)
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// Orders this thread's earlier generic-proxy accesses (plain loads/stores, acquire loads) with later accesses
-// through the asynchronous proxy (TMA), and the other way round.
 // Orders this thread's accesses through the generic proxy against its accesses through the asynchronous proxy (TMA), for
 // one state space only: the unqualified fence costs over a thousand cycles wherever it stands.
 __device__ __forceinline__ void fence_proxy_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -397,9 +397,9 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
     const uint32_t bar_acc_empty = bar_acc_full + 16;           // 2 x 8 B (used in the leader)
     const uint32_t bar_ring_full = bar_acc_empty + 16;          // RING x 8 B
     const uint32_t bar_ring_empty = bar_ring_full + 8 * RING;   // RING x 8 B (used in the leader)
-    const uint32_t bar_stg_full = bar_ring_empty + 8 * RING;    // staging buffer written (one arrival per epilogue warp)
-    const uint32_t bar_stg_empty = bar_stg_full + 8;            // staging buffer read by the stores (store warp)
-    const uint32_t tmem_slot = bar_stg_empty + 8;               // 4 B + abort flag 4 B + 8 B pad
+    const uint32_t bar_stg_full = bar_ring_empty + 8 * RING;    // 2 x 8 B: a 64-column half of the staging buffer written (its 4 warps)
+    const uint32_t bar_stg_empty = bar_stg_full + 16;           // 2 x 8 B: that half read by its store (store warp)
+    const uint32_t tmem_slot = bar_stg_empty + 16;              // 4 B + abort flag 4 B + 8 B pad
     const uint32_t ring_items = tmem_slot + 16;                 // RING x 16 B
     // items per matrix of the phases before phase q (q = 0 .. P): phase q has phase_first[q + 1] - phase_first[q] items
     volatile unsigned int* phase_first = reinterpret_cast<volatile unsigned int*>(smem_raw + (ring_items + 16 * RING - smem_u32(smem_raw)));   // (NS_MAX_PHASES + 1) x 4 B
@@ -424,8 +424,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         for (int s = 0; s < NENT; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(bar_acc_full + 8 * a, 1); mbar_init(bar_acc_empty + 8 * a, 2 * TC_EPI_WARPS); }
         for (int r = 0; r < RING; ++r) { mbar_init(bar_ring_full + 8 * r, 1); mbar_init(bar_ring_empty + 8 * r, RING_READERS); }
-        mbar_init(bar_stg_full, TC_EPI_WARPS);
-        mbar_init(bar_stg_empty, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_stg_full + 8 * b, TC_EPI_WARPS / 2); mbar_init(bar_stg_empty + 8 * b, 1); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         #pragma unroll
         for (int i = 0; i < NS_MAPS; ++i) asm volatile("prefetch.tensormap [%0];" ::"l"(&maps.m[i]) : "memory");
@@ -654,22 +653,33 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const CUtensorMap* tma_d = &maps.m[p.d_map + NS_TENSORS];     // 64 columns x 128 rows per store
                 const TileCoord tc = decode_tile(p, it.t);
                 const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
+                // The two 64-column halves of the staging buffer are separate buffers with their own barriers, filled by
+                // different warps.  A half is handed back when its own store has read it, and that is waited for only
+                // after the store of the other half has been issued: the engine reads one half while the other is written.
+                bool pending = false;
                 for (int u = 0; u < tc.nsub && ok; ++u) {
                     for (int ph = 0; ph < 2 && ok; ++ph) {
                         const int x0 = (tc.tn + u) * TC_BN + ph * EPI_COLS;
                         if (x0 >= p.N) continue;
                         if (!MONA_IN_BOUNDS(m0 < p.M + CTA_M && it.c < g.C && tc.tm < p.tiles_m, status, 106)) { ok = false; break; }
-                        if (!(ok = mbar_wait(bar_stg_full, staged & 1u, abort_flag, status, 13, TRACE_PTR(w_stg)))) break;
-                        ++staged;
                         #pragma unroll
                         for (int bx = 0; bx < 2; ++bx) {
+                            if (!(ok = mbar_wait(bar_stg_full + 8 * bx, staged & 1u, abort_flag, status, 13, TRACE_PTR(w_stg)))) break;
                             const int x = x0 + bx * TC_BOX;
                             if (x < p.N && m0 < p.M) tma_store_3d(tma_d, epi_buf + bx * 2 * BOX_BYTES, x, m0, it.c);   // clipped at the extents
+                            bulk_commit();
+                            if (pending) {
+                                bulk_wait_read<1>();       // the store before this one has read its half: its warps may refill it
+                                mbar_arrive_local(bar_stg_empty + 8 * (bx ^ 1));
+                            }
+                            pending = true;
                         }
-                        bulk_commit();
-                        bulk_wait_read();                  // the stores have read the buffer: the epilogue may refill it
-                        mbar_arrive_local(bar_stg_empty);
+                        ++staged;
                     }
+                }
+                if (ok && pending) {
+                    bulk_wait_read<0>();
+                    mbar_arrive_local(bar_stg_empty + 8);      // the last store of an item is always that of the second half
                 }
                 if (!ok) break;
                 bulk_wait_all();                           // the item's output is in global memory
@@ -778,7 +788,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
         bool alive = true;
         // 128 packed columns of this thread's row go to the staging buffer; the store warp sends them on
         auto put_phase = [&](const uint4* pk) -> bool {
-            if (!mbar_wait(bar_stg_empty, (staged & 1u) ^ 1u, abort_flag, status, 11, TRACE_PTR(w_stge))) return false;   // the previous phase has been read
+            if (!mbar_wait(bar_stg_empty + 8 * half, (staged & 1u) ^ 1u, abort_flag, status, 11, TRACE_PTR(w_stge))) return false;   // the previous phase of this half has been read
             if (!MONA_IN_BOUNDS(stage_off + 128u <= EPI_BUF_BYTES, status, 104)) return false;
             #pragma unroll
             for (int q = 0; q < 8; ++q) {
@@ -787,7 +797,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             }
             fence_proxy_async_shared();            // generic-proxy writes above must be visible to the TMA engine
             __syncwarp();
-            if (lane == 0) mbar_arrive_local(bar_stg_full);
+            if (lane == 0) mbar_arrive_local(bar_stg_full + 8 * half);
             ++staged;
             return true;
         };
