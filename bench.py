@@ -58,13 +58,33 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+_POWER_FIELD = None
+
+
+def power_field(index: int) -> str:
+    """`power.draw.instant` where this driver's nvidia-smi knows it (power.draw is a one-second average), else `power.draw`."""
+    global _POWER_FIELD
+    if _POWER_FIELD is None:
+        _POWER_FIELD = "power.draw"
+        try:
+            r = subprocess.run(["nvidia-smi", f"--id={index}", "--query-gpu=power.draw.instant", "--format=csv,noheader,nounits"],
+                               capture_output=True, text=True, timeout=20)
+            if r.returncode == 0:
+                float(r.stdout.strip().splitlines()[0])
+                _POWER_FIELD = "power.draw.instant"
+        except Exception:
+            pass
+    return _POWER_FIELD
+
+
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """Samples SM clock, board power and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,{power},clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index = index
+        self.Q = ClockSampler.Q.format(power=power_field(index))
         self.rows = []
         self.proc = None
         self.thread = None
@@ -107,7 +127,34 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "power_w_median": statistics.median(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def sustained(torch, dev, index, fn, flops_per_call, seconds=2.5):
+    """Runs fn() back to back for about `seconds` with clock and power sampling: sustained TFLOP/s, median watts and
+    clock over the window (its first 0.5 s left out of the medians), and joules per TFLOP."""
+    fn()
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(index)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    calls = 0
+    e0.record()
+    while time.time() - t0 < seconds:
+        fn()
+        calls += 1
+        if calls % 4 == 0:
+            torch.cuda.synchronize(dev)      # keep the host a few calls ahead at most, so the window is what was asked for
+    e1.record()
+    torch.cuda.synchronize(dev)
+    t1 = time.time()
+    c = sampler.stop(t0 + 0.5, t1)
+    tflops = flops_per_call * calls / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    w = c.get("power_w_median")
+    return {"tflops": tflops, "watts_median": w, "sm_mhz_median": c.get("sm_mhz"), "samples": c.get("samples"),
+            "reasons": c.get("reasons"), "joules_per_tflop": (w / tflops) if w and tflops else None, "seconds": t1 - t0}
 
 
 def oracle_sample(wl, budget_s: float = 12.0):
@@ -191,10 +238,11 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def library_yardstick(torch, dev, wl, chunk_budget=768 << 20):
+def library_yardstick(torch, dev, wl, chunk_budget=768 << 20, index=None):
     """Diagnostic only (never on the product path): the library batched GEMM (torch.bmm, bf16) on the three GEMM
     shapes of the workload's dominant bucket, one chunk's worth of matrices, timed back to back with CUDA events.
-    Dense products: the library computes all of X X^T and A A, not their lower triangles."""
+    Dense products: the library computes all of X X^T and A A, not their lower triangles.  With `index` (the device's
+    nvidia-smi index) the three products are also run back to back for a few seconds with power sampling."""
     best = None
     for sp in wl.specs:
         s_, l_ = min(sp.rows, sp.cols), max(sp.rows, sp.cols)
@@ -226,6 +274,12 @@ def library_yardstick(torch, dev, wl, chunk_budget=768 << 20):
     f1, f2, f3 = 2.0 * C * s_ * s_ * l_, 2.0 * C * s_ ** 3, 2.0 * C * s_ * s_ * l_
     out = {"shape": f"{C} x ({s_} x {l_})", "what": "torch.bmm bf16, dense products, back to back",
            "XXt": f1 / t1 / 1e12, "AA": f2 / t2 / 1e12, "BX": f3 / t3 / 1e12, "all_three": (f1 + f2 + f3) / (t1 + t2 + t3) / 1e12}
+    if index is not None:
+        def three():
+            torch.bmm(X, X.transpose(1, 2), out=A2)
+            torch.bmm(A, A, out=A2)
+            torch.bmm(A, X, out=Xn)
+        out["sustained"] = sustained(torch, dev, index, three, f1 + f2 + f3)
     del X, A, Xn, A2
     return out
 
@@ -372,6 +426,17 @@ def run_workload(torch, pkg, synth, shard, args, dev, local_rank, rank, world, d
                 "sm_mhz_during_pass": mhz, "clock_reasons_during_pass": (ns_clocks or {}).get("reasons"),
                 "util_per_clock": (ns_tflops / (2250.0 * mhz / 1965.0)) if mhz else None,
                 "util_per_clock_note": "achieved / (2250 TFLOP/s x median SM MHz during the pass / 1965)"}
+    if full and world == 1 and not args.no_yardstick:
+        # Diagnostic: the Newton-Schulz pass back to back for a few seconds with power sampling, to put joules per executed
+        # TFLOP beside the library's on the same shapes (main() adds that leg).  Runs after every timed figure above.
+        try:
+            roofline["energy"] = {"ns_kernel": sustained(torch, dev, local_rank, lambda: opt.step_ex(hp, params, gp.grads, None, 2), flops_exec),
+                                  "power_field": power_field(local_rank),
+                                  "note": "Newton-Schulz pass (executed flops) and the library's dense products of the dominant bucket, "
+                                          "each run back to back for ~2.5 s; watts = median nvidia-smi sample after the first 0.5 s"}
+            opt.poll_status()
+        except Exception as exc:
+            roofline["energy"] = {"error": str(exc)[:200]}
     result["roofline"] = roofline
     result.update({"opt": opt, "params": params, "gp": gp, "stream": stream, "barrier": barrier})
     return result
@@ -480,7 +545,10 @@ def main():
     wl, opt, params, gp, stream, barrier, hp = r["wl"], r["opt"], r["params"], r["gp"], r["stream"], r["barrier"], r["hp"]
     if rank == 0 and world == 1 and not args.no_yardstick:
         try:
-            r["roofline"]["library_same_shape_tflops"] = library_yardstick(torch, dev, wl, int(r["options"].chunk_budget_bytes))
+            lib = library_yardstick(torch, dev, wl, int(r["options"].chunk_budget_bytes), index=local_rank)
+            r["roofline"]["library_same_shape_tflops"] = lib
+            if lib and "sustained" in lib and isinstance(r["roofline"].get("energy"), dict) and "ns_kernel" in r["roofline"]["energy"]:
+                r["roofline"]["energy"]["library_same_shape"] = lib.pop("sustained")
         except Exception as exc:     # a diagnostic must not take the benchmark down (e.g. no memory left for its operands)
             r["roofline"]["library_same_shape_tflops"] = {"error": str(exc)[:200]}
 
