@@ -241,6 +241,17 @@ mona_status mona_last_ns_flops(const mona_handle* h, double* executed, double* d
  * 3 s^2 l + s^3 per matrix and iteration (tensor-core path only). */
 mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful);
 
+/* The order in which the Newton-Schulz kernel hands out its work items (tiles), computed on the HOST with the cursor
+ * the kernel's scheduler uses; no device is needed.  The paper has no counterpart: this exposes the property the
+ * kernel's freedom from deadlock rests on - every item comes after all items it depends on (GEMM q of a matrix after
+ * all items of GEMM q - 1 of that matrix) - so that it can be tested for any launch shape.
+ *   n_matrices, n_phases (1..15), delay (>= 1, see mona_options.ns_delay), items_per_phase[n_phases]: items per matrix.
+ * Writes (matrix, phase, item) triples of the items start, start + stride, start + 2 stride, ... (one CTA pair sees such
+ * a subsequence) into the HOST array out_cqt (3 int32 per item), at most `capacity` items; *n_written receives the
+ * count.  MONA_ERR_INVALID_ARG for null pointers or non-positive sizes. */
+mona_status mona_work_order(int32_t n_matrices, int32_t n_phases, int32_t delay, const uint32_t* items_per_phase,
+                            uint32_t start, uint32_t stride, int32_t* out_cqt, size_t capacity, size_t* n_written);
+
 /* Profiling build only (library compiled with -DMONA_TRACE; every other build returns MONA_ERR_NOT_BUILT and
  * touches nothing).  The paper has no counterpart: this is the instrument behind the per-role wait times quoted
  * for the Newton-Schulz kernel.  In that build every role of the kernel (TMA producer, MMA issuer, scheduler,

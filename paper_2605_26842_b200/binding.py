@@ -65,6 +65,8 @@ def lib() -> C.CDLL:
     L.mona_create_opt.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, C.POINTER(Options), vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_last_ns_useful_flops.argtypes = [vp, C.POINTER(C.c_double)]
     L.mona_trace_read.argtypes = [C.POINTER(C.c_ulonglong), C.c_size_t, C.c_int]
+    L.mona_work_order.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_uint32), C.c_uint32, C.c_uint32,
+                                  C.POINTER(C.c_int32), C.c_size_t, C.POINTER(C.c_size_t)]
     L.mona_create.argtypes = [C.POINTER(vp), C.POINTER(MatrixDesc), C.c_int64, vp, C.c_size_t, vp, C.c_size_t, C.c_int]
     L.mona_step.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vp]
     L.mona_step_ex.argtypes = [vp, C.POINTER(Hparams), vpp, vpp, vpp, C.c_uint32, vp]
@@ -82,10 +84,24 @@ def lib() -> C.CDLL:
     L.mona_destroy.restype = None
     for name in ("mona_default_hparams", "mona_set_chunk_budget", "mona_set_chunk_overlap", "mona_query_sizes", "mona_create", "mona_step",
                  "mona_step_ex", "mona_step_host", "mona_poll_status", "mona_state_layout", "mona_last_ns_flops",
-                 "mona_default_options", "mona_query_sizes_opt", "mona_create_opt", "mona_last_ns_useful_flops", "mona_trace_read"):
+                 "mona_default_options", "mona_query_sizes_opt", "mona_create_opt", "mona_last_ns_useful_flops", "mona_trace_read", "mona_work_order"):
         getattr(L, name).restype = C.c_int
     _lib = L
     return L
+
+
+def work_order(n_matrices: int, delay: int, items_per_phase: Sequence[int], start: int = 0, stride: int = 1, capacity: Optional[int] = None):
+    """mona_work_order(): (matrix, phase, item) of the kernel's work items start, start + stride, ... as a list of tuples."""
+    P = len(items_per_phase)
+    if capacity is None:
+        capacity = (n_matrices * sum(items_per_phase) - start + stride - 1) // stride if n_matrices * sum(items_per_phase) > start else 0
+    ipp = (C.c_uint32 * max(1, P))(*items_per_phase)
+    out = (C.c_int32 * (3 * max(1, capacity)))()
+    n = C.c_size_t(0)
+    st = lib().mona_work_order(n_matrices, P, delay, ipp, start, stride, out, capacity, C.byref(n))
+    if st:
+        raise MonaError(st, "mona_work_order")
+    return [(out[3 * i], out[3 * i + 1], out[3 * i + 2]) for i in range(n.value)]
 
 
 def trace_read(reset: bool = True, rows: int = TRACE_ROWS):

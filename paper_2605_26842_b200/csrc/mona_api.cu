@@ -724,6 +724,15 @@ static_assert(MONA_TRACE_ROWS == mona::NS_TRACE_ROWS && MONA_TRACE_SLOTS == mona
               (int)MONA_TRACE_EPI_ROLE == (int)mona::NS_TRACE_EPI_ROLE && (int)MONA_TRACE_SCHED_ROLE == (int)mona::NS_TRACE_SCHED_ROLE,
               "the public description of the profiling table follows the kernel's");
 
+mona_status mona_work_order(int32_t n_matrices, int32_t n_phases, int32_t delay, const uint32_t* items_per_phase,
+                            uint32_t start, uint32_t stride, int32_t* out_cqt, size_t capacity, size_t* n_written) {
+    if (!n_written) return MONA_ERR_INVALID_ARG;
+    const int n = mona::ns_work_order(n_matrices, n_phases, delay, items_per_phase, start, stride, out_cqt, capacity);
+    if (n < 0) return MONA_ERR_INVALID_ARG;
+    *n_written = (size_t)n;
+    return MONA_OK;
+}
+
 mona_status mona_trace_read(unsigned long long* out, size_t rows, int reset) {
     if (rows && !out) return MONA_ERR_INVALID_ARG;
     int available = 0;

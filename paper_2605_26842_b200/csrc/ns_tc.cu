@@ -696,35 +696,14 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             // ---------------- scheduler (leader CTA only) ----------------
             const uint32_t ring_items_peer = map_to_cta(ring_items, 1), ring_full_peer = map_to_cta(bar_ring_full, 1);
             const uint32_t ring_full_own = map_to_cta(bar_ring_full, 0);
-            // Item order: for tau = 0, 1, ...: for q = 0 .. P-1: the items of phase q of matrix c = tau - delay * q, where that
-            // matrix exists, i.e. for q_lo(tau) <= q <= q_hi(tau) with q_hi = min(P - 1, tau / delay) (c >= 0) and
-            // q_lo = ceil((tau - C + 1) / delay) (c < C).  The cursor (tau, index of the first item of its group of phases)
-            // only moves forward, a whole tau at a time; q_lo and q_hi are kept incrementally, so that finding an item costs
-            // a few shared-memory reads however many items the other pairs have taken since this pair's last one.
-            const int C = g.C, delay = g.delay;
-            int cur_tau = 0, q_lo = 0, q_hi = 0, lo_cnt = 0, hi_cnt = 0;
-            unsigned cur_base = 0;
+            // The item order and the cursor that walks it are NsItemCursor's (ns_tc.cuh); per-phase item counts come from
+            // shared memory.
+            NsItemCursor cursor(g.C, P, g.delay);
             auto decode = [&](unsigned idx, Item& it) -> bool {
                 it.stop = idx >= g.total_items ? 1 : 0;
                 it.c = it.q = it.t = 0;
                 if (it.stop) return true;
-                while (true) {
-                    const unsigned n_tau = q_lo <= q_hi ? phase_first[q_hi + 1] - phase_first[q_lo] : 0u;
-                    if (idx < cur_base + n_tau) break;
-                    if (cur_tau >= C + P * delay) return false;          // past the last group: the item count and this walk disagree
-                    cur_base += n_tau;
-                    ++cur_tau;
-                    if (++hi_cnt == delay) { hi_cnt = 0; if (q_hi < P - 1) ++q_hi; }
-                    if (cur_tau == C) { q_lo = 1; lo_cnt = 0; }
-                    else if (cur_tau > C && ++lo_cnt == delay) { lo_cnt = 0; ++q_lo; }
-                }
-                const unsigned r = idx - cur_base + phase_first[q_lo];      // counted from phase 0 of this tau
-                int q = q_lo;
-                while (phase_first[q + 1] <= r) ++q;                        // ends at q <= q_hi since r < phase_first[q_hi + 1]
-                it.q = q;
-                it.t = (int)(r - phase_first[q]);
-                it.c = cur_tau - delay * q;
-                return true;
+                return cursor.find(idx, phase_first, it.c, it.q, it.t);      // false: the item count and the walk disagree
             };
             // The phase before an item must be complete for its matrix: its outputs are the item's operands, and the buffers
             // the item overwrites were last read two phases further back.
@@ -976,6 +955,23 @@ cudaError_t ns_trace_read(unsigned long long* out, size_t rows, int reset, int* 
     *available = 0;
     return cudaSuccess;
 #endif
+}
+
+int ns_work_order(int C, int P, int delay, const unsigned int* items_per_phase, unsigned start, unsigned stride, int* cqt,
+                  size_t capacity) {
+    if (C <= 0 || P <= 0 || P > NS_MAX_PHASES || delay <= 0 || !items_per_phase || stride == 0 || (capacity && !cqt)) return -1;
+    unsigned first[NS_MAX_PHASES + 1];
+    first[0] = 0u;
+    for (int q = 0; q < P; ++q) first[q + 1] = first[q] + items_per_phase[q];
+    const unsigned long long total = (unsigned long long)first[P] * (unsigned long long)C;
+    NsItemCursor cursor(C, P, delay);
+    size_t n = 0;
+    for (unsigned long long idx = start; idx < total && n < capacity; idx += stride, ++n) {
+        int c, q, t;
+        if (!cursor.find((unsigned)idx, first, c, q, t)) return -2;
+        cqt[3 * n] = c; cqt[3 * n + 1] = q; cqt[3 * n + 2] = t;
+    }
+    return (int)n;
 }
 
 void ns_phase_plan(NsPhase& p) {

@@ -70,6 +70,40 @@ struct NsProgram {
                                 //    report STATUS_TIMEOUT and leave cleanly (all copies still complete; nothing faults)
 };
 
+// The kernel's work order, as a cursor that only moves forward (host and device).
+//     for tau = 0, 1, ...: for q = 0 .. P-1: the items of phase q of matrix c = tau - delay * q, where that matrix exists,
+// i.e. for q_lo(tau) <= q <= q_hi(tau) with q_hi = min(P - 1, tau / delay) (c >= 0) and q_lo = ceil((tau - C + 1) / delay)
+// (c < C).  Phase q of matrix c therefore comes `delay` values of tau after phase q - 1 of the same matrix: every item follows
+// all items it depends on.  The cursor advances a whole tau at a time and keeps q_lo and q_hi incrementally, so finding an
+// item costs a few reads of `first` (no divisions) however many items lie between two calls.
+// `first[q]`, q = 0 .. P: items per matrix of the phases before phase q (first[0] = 0).
+struct NsItemCursor {
+    int C, P, delay;
+    int tau = 0, q_lo = 0, q_hi = 0, lo_cnt = 0, hi_cnt = 0;
+    unsigned base = 0;                  // index of the first item of the current tau
+    __host__ __device__ NsItemCursor(int C_, int P_, int delay_) : C(C_), P(P_), delay(delay_) {}
+    // Finds item `idx`, which must not be smaller than any index asked before.  False when the walk runs past the last
+    // group without reaching it (idx is not an item of the launch).
+    __host__ __device__ bool find(unsigned idx, const volatile unsigned int* first, int& c, int& q, int& t) {
+        while (true) {
+            const unsigned n_tau = q_lo <= q_hi ? first[q_hi + 1] - first[q_lo] : 0u;
+            if (idx < base + n_tau) break;
+            if (tau >= C + P * delay) return false;
+            base += n_tau;
+            ++tau;
+            if (++hi_cnt == delay) { hi_cnt = 0; if (q_hi < P - 1) ++q_hi; }
+            if (tau == C) { q_lo = 1; lo_cnt = 0; }
+            else if (tau > C && ++lo_cnt == delay) { lo_cnt = 0; ++q_lo; }
+        }
+        const unsigned r = idx - base + first[q_lo];       // counted from phase 0 of this tau
+        q = q_lo;
+        while (first[q + 1] <= r) ++q;                      // ends at q <= q_hi since r < first[q_hi + 1]
+        t = (int)(r - first[q]);
+        c = tau - delay * q;
+        return true;
+    }
+};
+
 // Layout of the profiling build's table (-DMONA_TRACE): one row per CTA (blockIdx.x; even rows are the leaders, which
 // alone run the MMA issuer and the scheduler), NS_TRACE_SLOTS 64-bit words per row, all in SM clock cycles unless noted,
 // summed over the launches since the last reset.
@@ -121,6 +155,11 @@ inline size_t ns_sched_words(int C, int P) { return 64 + (size_t)C * P; }
 // Sets the kernel's shared-memory attribute and finds how many CTA pairs the device holds at once.
 // Call once per device before the first launch.
 cudaError_t ns_configure(int* max_pairs);
+// Host-side walk of the work order of a launch over C matrices and P phases with `items_per_phase[q]` items per matrix:
+// writes (c, q, t) of the items start, start + stride, ... into `cqt` (3 ints per item, at most `capacity` items) with the
+// cursor the kernel's scheduler uses.  Returns the number written, -1 for bad arguments, -2 if the walk fails.
+int ns_work_order(int C, int P, int delay, const unsigned int* items_per_phase, unsigned start, unsigned stride, int* cqt,
+                  size_t capacity);
 // Copies the first `rows` rows of the profiling table to `out` (host) after synchronising the device, and clears the table
 // when `reset` is set.  *available = 0 (and nothing else happens) unless the library was built with -DMONA_TRACE.
 cudaError_t ns_trace_read(unsigned long long* out, size_t rows, int reset, int* available);
