@@ -281,10 +281,13 @@ typedef enum mona_trace_slot {
     MONA_TRACE_STORE_STAGED = 13,     /* store warp: waiting for a staged 128-column phase                     */
     MONA_TRACE_STORE_ROLE = 14,       /* store warp: whole role                                                */
     MONA_TRACE_ITEMS = 15,            /* work items completed by this CTA (a count, not cycles)                */
-    MONA_TRACE_TILE0 = 16             /* + 4 * kind + {0: cycles of the MMA issuer inside tiles of the kind, 1: their
+    MONA_TRACE_TILE0 = 16,            /* + 4 * kind + {0: cycles of the MMA issuer inside tiles of the kind, 1: their
                                          k-slices (a count), 2: of the cycles, waiting for operands, 3: waiting for an
                                          accumulator}; kind 0 / 1: X X^T off / on the diagonal, 2 / 3: b A + c A^2 + a I
                                          off / on the diagonal, 4: 256 x 512 macro-tile of X' = B' X, 5: single tile of it */
+    MONA_TRACE_EPI_TILE0 = 40         /* + 4 * kind + {0: cycles of an epilogue warp inside items of the kind, 1: items (a
+                                         count), 2: of the cycles, waiting for accumulators, 3: waiting for the staging
+                                         buffer}, sums over the 8 epilogue warps                                      */
 } mona_trace_slot;
 mona_status mona_trace_read(unsigned long long* out, size_t rows, int reset);
 

@@ -720,7 +720,7 @@ mona_status mona_last_ns_useful_flops(const mona_handle* h, double* useful) {
 }
 
 static_assert(MONA_TRACE_ROWS == mona::NS_TRACE_ROWS && MONA_TRACE_SLOTS == mona::NS_TRACE_SLOTS &&
-              (int)MONA_TRACE_TILE0 == (int)mona::NS_TRACE_TILE0 && (int)MONA_TRACE_ITEMS == (int)mona::NS_TRACE_ITEMS &&
+              (int)MONA_TRACE_TILE0 == (int)mona::NS_TRACE_TILE0 && (int)MONA_TRACE_EPI_TILE0 == (int)mona::NS_TRACE_EPI_TILE0 && (int)MONA_TRACE_ITEMS == (int)mona::NS_TRACE_ITEMS &&
               (int)MONA_TRACE_EPI_ROLE == (int)mona::NS_TRACE_EPI_ROLE && (int)MONA_TRACE_SCHED_ROLE == (int)mona::NS_TRACE_SCHED_ROLE,
               "the public description of the profiling table follows the kernel's");
 

@@ -786,6 +786,7 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
             __syncwarp();
             if (lane == 0) mbar_arrive_slot_read(ring_empty_leader + 8 * (n % RING), it.c, it.q, it.t, it.stop);   // every lane has its copy of the item
             if (it.stop) break;
+            TRACE_ONLY(const uint32_t t_item0 = trace_clock();)
             const NsPhase& p = g.ph[it.q];
             const TileCoord tc = decode_tile(p, it.t);
             const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
@@ -916,6 +917,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
 #ifdef MONA_TRACE
             if (lane == 0) {      // one lane per warp: the table holds sums over the eight epilogue warps
                 trace_add(NS_TRACE_EPI_RING, w_ring); trace_add(NS_TRACE_EPI_ACC_FULL, w_accf); trace_add(NS_TRACE_EPI_STAGE_EMPTY, w_stge);
+                const bool diag = p.ab_same && tc.tm == tc.tn && tc.nsub == 1;
+                const int kind = !p.symmetric ? (tc.nsub == 2 ? 4 : 5) : ((p.cin ? 2 : 0) + (diag ? 1 : 0));
+                const int slot = NS_TRACE_EPI_TILE0 + 4 * kind;
+                trace_add(slot, trace_clock() - t_item0); trace_add(slot + 1, 1u); trace_add(slot + 2, w_accf); trace_add(slot + 3, w_stge);
             }
             w_ring = w_accf = w_stge = 0;
 #endif

@@ -126,10 +126,13 @@ enum NsTraceSlot {
     NS_TRACE_STORE_STAGED = 13,     // store warp: waiting for a staged phase
     NS_TRACE_STORE_ROLE = 14,       // store warp: whole role
     NS_TRACE_ITEMS = 15,            // work items completed by this CTA (a count)
-    NS_TRACE_TILE0 = 16             // 6 kinds of tile x {cycles of the MMA issuer inside the tile, k-slices (a count), of which
+    NS_TRACE_TILE0 = 16,            // 6 kinds of tile x {cycles of the MMA issuer inside the tile, k-slices (a count), of which
                                     // waiting for operands, of which waiting for an accumulator}; kinds: 0/1 X X^T off/on the
                                     // diagonal, 2/3 b A + c A^2 + a I off/on the diagonal, 4 macro-tile and 5 single tile of X' = B' X
+    NS_TRACE_EPI_TILE0 = 40         // the same 6 kinds x {cycles of an epilogue warp inside items of the kind, items (a count), of
+                                    // which waiting for accumulators, of which waiting for the staging buffer}, sums over the 8 warps
 };
+static_assert(NS_TRACE_EPI_TILE0 + 4 * 6 <= NS_TRACE_SLOTS, "profiling table");
 
 struct alignas(64) NsMaps {
     CUtensorMap m[NS_MAPS];

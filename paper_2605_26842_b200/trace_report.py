@@ -95,6 +95,14 @@ def summarise(res):
     for v in tiles.values():
         v["share_of_issuer_time_pct"] = 100.0 * v["cycles_per_k_slice"] * v["k_slices"] / total
     out["tiles"] = tiles
+    epi = {}
+    for kind, label in enumerate(KINDS):
+        b = 40 + 4 * kind
+        cyc, n, wa, ws = (sum(r[b + j] for r in rows) for j in range(4))
+        if n:
+            epi[label] = {"items_per_warp": n / 8, "cycles_per_item": cyc / n, "waiting_accumulator": wa / n, "waiting_staging": ws / n,
+                          "working": (cyc - wa - ws) / n}
+    out["epilogue"] = epi
     issuer = mean(lead, 5)
     out["mma_issuer_inside_tiles_pct"] = 100.0 * total / len(lead) / issuer if issuer else 0.0
     return out
@@ -125,6 +133,10 @@ def main():
         print(f"    {label:<26s} {v['k_slices']:>9d} k-slices  {v['cycles_per_k_slice']:7.1f} cycles "
               f"(tensor peak {v['tensor_peak_cycles']:.0f}) = issuing {v['issuing']:6.1f} + operands {v['waiting_operands']:6.1f} "
               f"+ accumulator {v['waiting_accumulator']:6.1f};  {v['share_of_issuer_time_pct']:4.1f} % of the time inside tiles")
+    print("  per work item of an epilogue warp, SM cycles (a CTA's 128 rows of the tile or macro-tile):")
+    for label, v in s["epilogue"].items():
+        print(f"    {label:<26s} {v['cycles_per_item']:8.0f} cycles = working {v['working']:6.0f} + accumulator {v['waiting_accumulator']:6.0f} "
+              f"+ staging buffer {v['waiting_staging']:6.0f}")
     return 0 if s["status"] == 0 else 1
 
 
