@@ -372,6 +372,12 @@ __device__ __forceinline__ void ld8(const float* p, float* v) {
                  : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
                  : "l"(p));
 }
+// 32 bytes of bf16 data written earlier in this launch by other CTAs: from L2 (.cg), never from a line L1 may still hold
+__device__ __forceinline__ void ld8cg(const void* p, uint32_t* w) {
+    asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(p));
+}
 __device__ __forceinline__ void st8(float* p, const float* v) {
     asm volatile("st.global.cs.v8.f32 [%8], {%0, %1, %2, %3, %4, %5, %6, %7};"
                  ::"f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "l"(p)
@@ -840,15 +846,30 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const uint32_t acc = acc0 + u;
                 const int n0 = (tc.tn + u) * TC_BN;
                 const int nphases = (p.N - n0 > EPI_COLS) ? 2 : 1;
-                // operand of the axpy term, requested before the accumulator is ready.  It was written by other CTAs of this
-                // launch, so it is read from L2 (ld.cg), never from a line L1 may still hold from an earlier iteration.
-                uint4 cin_raw[8];
+                // Operand of the axpy term: this thread's 64 values of a phase (128 bytes), requested before the accumulator is
+                // ready (first phase) or before the previous phase is staged (second), so that the round trip is hidden.  It was written by other CTAs of this
+                // launch, so it is read from L2 (.cg), never from a line L1 may still hold from an earlier iteration.  A thread
+                // owns a row, so a warp's load touches 32 lines whatever its width: 32-byte accesses halve the requests.
+                uint32_t cin_w[32];
+                const bool cin_v8 = p.cin && ((p.ld | p.mat_stride | (long long)p.N) & 15) == 0 && (reinterpret_cast<uintptr_t>(p.cin) & 31) == 0;
                 auto load_cin = [&](int ph) {
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
-                    #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (row_ok && gc0 + 8 * q < p.N && MONA_IN_BOUNDS(row_off + gc0 + 8 * q + 8 <= (long long)g.C * p.mat_stride, status, 105)) cin_raw[q] = __ldcg(reinterpret_cast<const uint4*>(p.cin + row_off + gc0 + 8 * q));
-                        else cin_raw[q] = make_uint4(0u, 0u, 0u, 0u);
+                    if (cin_v8) {
+                        #pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (row_ok && gc0 + 16 * q < p.N && MONA_IN_BOUNDS(row_off + gc0 + 16 * q + 16 <= (long long)g.C * p.mat_stride, status, 105)) ld8cg(p.cin + row_off + gc0 + 16 * q, cin_w + 8 * q);
+                            else {
+                                #pragma unroll
+                                for (int j = 0; j < 8; ++j) cin_w[8 * q + j] = 0u;
+                            }
+                        }
+                    } else {
+                        #pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            uint4 r = make_uint4(0u, 0u, 0u, 0u);
+                            if (row_ok && gc0 + 8 * q < p.N && MONA_IN_BOUNDS(row_off + gc0 + 8 * q + 8 <= (long long)g.C * p.mat_stride, status, 105)) r = __ldcg(reinterpret_cast<const uint4*>(p.cin + row_off + gc0 + 8 * q));
+                            cin_w[4 * q] = r.x; cin_w[4 * q + 1] = r.y; cin_w[4 * q + 2] = r.z; cin_w[4 * q + 3] = r.w;
+                        }
                     }
                 };
                 if (p.cin) load_cin(0);
@@ -869,16 +890,10 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                     }
                     const int gc0 = n0 + ph * EPI_COLS + half * 64;
                     if (p.cin) {
-                        const uint32_t w[32] = {cin_raw[0].x, cin_raw[0].y, cin_raw[0].z, cin_raw[0].w, cin_raw[1].x, cin_raw[1].y,
-                                                cin_raw[1].z, cin_raw[1].w, cin_raw[2].x, cin_raw[2].y, cin_raw[2].z, cin_raw[2].w,
-                                                cin_raw[3].x, cin_raw[3].y, cin_raw[3].z, cin_raw[3].w, cin_raw[4].x, cin_raw[4].y,
-                                                cin_raw[4].z, cin_raw[4].w, cin_raw[5].x, cin_raw[5].y, cin_raw[5].z, cin_raw[5].w,
-                                                cin_raw[6].x, cin_raw[6].y, cin_raw[6].z, cin_raw[6].w, cin_raw[7].x, cin_raw[7].y,
-                                                cin_raw[7].z, cin_raw[7].w};
                         #pragma unroll
                         for (int h = 0; h < 32; ++h) {
-                            v[2 * h] = fmaf(c1, __uint_as_float(w[h] << 16), c2 * v[2 * h]);
-                            v[2 * h + 1] = fmaf(c1, __uint_as_float(w[h] & 0xffff0000u), c2 * v[2 * h + 1]);
+                            v[2 * h] = fmaf(c1, __uint_as_float(cin_w[h] << 16), c2 * v[2 * h]);
+                            v[2 * h + 1] = fmaf(c1, __uint_as_float(cin_w[h] & 0xffff0000u), c2 * v[2 * h + 1]);
                         }
                         if (ph + 1 < nphases) load_cin(ph + 1);
                     } else {
