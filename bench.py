@@ -33,7 +33,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised in profiles/ns_chunk_kernel_moe7b_1L.md: the launch over a 93-matrix 768x2048 chunk, the launch shape that
 # makes up most of the default workload (40 of its 56 launches per step are of this shape or its tall twin).  Valid only
 # for the kernel source the counters were taken with (hash of ns_tc.cu + ns_tc.cuh).
-NCU_TRAFFIC = {"source_sha256_16": "4e19e59a3ea7fac1", "bytes_per_launch": 6.674e9,
+NCU_TRAFFIC = {"source_sha256_16": "d420627d482a0ead", "bytes_per_launch": 6.690e9,
                "unit": "DRAM bytes of one launch over a 93-matrix 768x2048 chunk (ncu; 2.153 TFLOP executed in that launch)"}
 
 

@@ -660,9 +660,8 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                 const TileCoord tc = decode_tile(p, it.t);
                 const int m0 = tc.tm * TC_BM + (int)rank * CTA_M;
                 // The two 64-column halves of the staging buffer are separate buffers with their own barriers, filled by
-                // different warps.  A half is handed back when its own store has read it, and that is waited for only
-                // after the store of the other half has been issued: the engine reads one half while the other is written.
-                bool pending = false;
+                // different warps: each half is stored as soon as it is full and handed back as soon as its own store has
+                // read it, the first half while the second store is still reading.
                 for (int u = 0; u < tc.nsub && ok; ++u) {
                     for (int ph = 0; ph < 2 && ok; ++ph) {
                         const int x0 = (tc.tn + u) * TC_BN + ph * EPI_COLS;
@@ -674,18 +673,14 @@ ns_chunk_kernel(const __grid_constant__ NsMaps maps, const __grid_constant__ NsP
                             const int x = x0 + bx * TC_BOX;
                             if (x < p.N && m0 < p.M) tma_store_3d(tma_d, epi_buf + bx * 2 * BOX_BYTES, x, m0, it.c);   // clipped at the extents
                             bulk_commit();
-                            if (pending) {
-                                bulk_wait_read<1>();       // the store before this one has read its half: its warps may refill it
-                                mbar_arrive_local(bar_stg_empty + 8 * (bx ^ 1));
-                            }
-                            pending = true;
                         }
+                        if (!ok) break;
+                        bulk_wait_read<1>();               // the first store has read its half: its warps may refill it
+                        mbar_arrive_local(bar_stg_empty);
+                        bulk_wait_read<0>();
+                        mbar_arrive_local(bar_stg_empty + 8);
                         ++staged;
                     }
-                }
-                if (ok && pending) {
-                    bulk_wait_read<0>();
-                    mbar_arrive_local(bar_stg_empty + 8);      // the last store of an item is always that of the second half
                 }
                 if (!ok) break;
                 bulk_wait_all();                           // the item's output is in global memory
