@@ -607,7 +607,7 @@ def main():
     others = None
     if world == 1 and not args.no_others and args.config == 3 and args.layers is None:
         others = {}
-        for idx in (1, 2, 4):
+        for idx in (1, 2, 4, 5):       # 5: the paper-shaped 256 x 768 expert set (its smallest model's experts)
             try:
                 o = run_workload(torch, pkg, synth, shard, args, dev, local_rank, rank, world, dist, idx, None, 3, 3, full=False)
                 ph = o["phases"]
