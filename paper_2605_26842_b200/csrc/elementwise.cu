@@ -257,7 +257,28 @@ update_kernel(ChunkPtrs ptrs, const OT* __restrict__ O, long long e, long long s
     float* __restrict__ Oout = ptrs.o[c];
     const OT* __restrict__ Oc = O + (long long)c * e;
     if (VEC == 4) {
-        for (long long i = lo + (long long)threadIdx.x * 4; i < hi; i += (long long)EW_THREADS * 4) {
+        // Four independent vectors per thread and trip, all loads first: when the block runs squeezed beside a resident
+        // GEMM CTA (one 128-thread block per SM), the bytes it keeps in flight are all the bandwidth it gets.
+        constexpr int UNROLL = 4;
+        constexpr long long STEP = (long long)EW_THREADS * 4;
+        long long i = lo + (long long)threadIdx.x * 4;
+        for (; i + (UNROLL - 1) * STEP < hi; i += UNROLL * STEP) {
+            float4 w[UNROLL], o[UNROLL];
+            #pragma unroll
+            for (int u = 0; u < UNROLL; ++u) w[u] = __ldcs(reinterpret_cast<const float4*>(W + i + u * STEP));
+            #pragma unroll
+            for (int u = 0; u < UNROLL; ++u) o[u] = GradLoad<OT>::load4(Oc + i + u * STEP);
+            #pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                w[u].x = fmaf(-eta_gamma, o[u].x, fmaf(-eta_lambda, w[u].x, w[u].x));
+                w[u].y = fmaf(-eta_gamma, o[u].y, fmaf(-eta_lambda, w[u].y, w[u].y));
+                w[u].z = fmaf(-eta_gamma, o[u].z, fmaf(-eta_lambda, w[u].z, w[u].z));
+                w[u].w = fmaf(-eta_gamma, o[u].w, fmaf(-eta_lambda, w[u].w, w[u].w));
+                __stcs(reinterpret_cast<float4*>(W + i + u * STEP), w[u]);
+                if (Oout) *reinterpret_cast<float4*>(Oout + i + u * STEP) = o[u];
+            }
+        }
+        for (; i < hi; i += STEP) {
             float4 w = __ldcs(reinterpret_cast<const float4*>(W + i));
             float4 o = GradLoad<OT>::load4(Oc + i);
             w.x = fmaf(-eta_gamma, o.x, fmaf(-eta_lambda, w.x, w.x));
