@@ -120,9 +120,10 @@ class ClockSampler:
             if len(f) < 7:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+                vals = (float(f[0]), float(f[1]), float(f[2]))
             except ValueError:
                 continue
+            sm.append(vals[0]); mx.append(vals[1]); power.append(vals[2])
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
