@@ -164,6 +164,14 @@ def test_many_small_matrices_span_several_chunks():
     check(errs, TOL_O_BF16)
 
 
+def test_a_layer_of_paper_shaped_experts_in_both_orientations():
+    """128 + 128 experts of 256 x 768 and 768 x 256 (the expert shape of the paper's smallest model): every product of such
+    a matrix is one or three tiles of 4 or 12 k-slices, so the launch is thousands of short items bound by their
+    epilogues; sampled matrices are followed by the oracle."""
+    errs = run_case([(128, 256, 768), (128, 768, 256)], steps=2, seed=31, sample={0: [0, 63, 127], 1: [0, 64, 127]})
+    check(errs, TOL_O_BF16)
+
+
 def test_fixed_scale_and_other_hyperparameters():
     hp = pkg.default_hparams(scale_mode=1, scale_value=0.37, lr=5e-3, momentum=0.8, weight_decay=0.0,
                              accel_beta=0.9, accel_alpha=-5.0)
